@@ -1,0 +1,144 @@
+/*
+ * lrsa.h - C ABI of the B200 (sm_100a) Lag-Relative Sparse Attention library.
+ *
+ * The library computes the data-parallel hot path of LRSA post-training:
+ *   1. lrsa_score_select : LagKV token scores (Section 3.2, Eq. 4-8) and the top-K kept
+ *                          positions of every lag window (text after Eq. 8),
+ *   2. lrsa_attn_fwd     : masked softmax attention (Section 3.1, Eq. 3) under the static
+ *                          chunked mask of Section 3.2 (Attn-Fill 1 / Attn-Fill 2),
+ *   3. lrsa_attn_bwd     : its gradient with the mask held constant.
+ *
+ * Conventions common to every call
+ * --------------------------------
+ * Tensors  : row-major, contiguous, bf16 unless stated.  Q, O, dO, dQ are [batch, n_q_heads,
+ *            seq_len, head_dim]; K, V, dK, dV are [batch, n_kv_heads, seq_len, head_dim].
+ *            Query head h uses KV head h / (n_q_heads / n_kv_heads).
+ * Pointers : every tensor/workspace pointer is a DEVICE pointer owned by the caller, aligned to
+ *            16 bytes (workspace: 256 bytes).  `params` is a HOST pointer.  The library
+ *            allocates no device memory and keeps no state between calls.
+ * Geometry : positions [0, S) are sinks.  Window w covers [S + w*L, S + (w+1)*L).
+ *            W = floor((N-S)/L) full windows, tail T = N - S - W*L (< L) tokens.
+ *            W_sel = max(W-1, 0) windows have a full following window and are scored.
+ * Stream   : `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
+ *            enqueue work and return without synchronising.  Two calls that use the same
+ *            workspace must be ordered (same stream, or otherwise serialised).
+ * Errors   : the int return value is an lrsa_status.  All argument checks happen on the host
+ *            before anything is enqueued; on a non-zero status nothing was launched, except
+ *            LRSA_ERR_CUDA which reports a launch failure of the CUDA runtime.
+ *            Device-side waits are bounded; if one expires the kernel records it in the
+ *            workspace and lrsa_workspace_status returns LRSA_ERR_TIMEOUT (outputs are
+ *            then undefined).
+ */
+#ifndef LRSA_H_
+#define LRSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum lrsa_status {
+  LRSA_OK = 0,
+  LRSA_ERR_INVALID_ARG = 1,         /* null pointer, non-positive size, K > L, Hq % Hkv != 0, misaligned */
+  LRSA_ERR_UNSUPPORTED = 2,         /* head_dim not in {64,128}, chunk != lag, seq_len < n_sink, ... */
+  LRSA_ERR_WORKSPACE_TOO_SMALL = 3,
+  LRSA_ERR_CUDA = 4,                /* CUDA runtime error while enqueueing */
+  LRSA_ERR_TIMEOUT = 5              /* a bounded device-side wait expired */
+} lrsa_status;
+
+typedef struct lrsa_params {
+  int32_t batch;         /* B >= 1 */
+  int32_t n_q_heads;     /* Hq, multiple of n_kv_heads (GQA) */
+  int32_t n_kv_heads;    /* Hkv */
+  int32_t seq_len;       /* N >= n_sink */
+  int32_t head_dim;      /* d in {64, 128} */
+  int32_t chunk;         /* query chunk size; must equal lag */
+  int32_t lag;           /* L, lag window size */
+  int32_t top_k;         /* K = r*L kept tokens per window, 1 <= K <= L */
+  int32_t n_sink;        /* S >= 0 */
+  int32_t n_dense_prev;  /* 1: the window just before the query chunk is seen uncompressed (the
+                            paper's "sliding window"); 0: it is compressed too when scored */
+  int32_t std_ddof;      /* divisor of the per-token Std is head_dim - std_ddof; 0 or 1 */
+  float softmax_scale;   /* 0 -> 1/sqrt(head_dim) as in Eq. 3 */
+} lrsa_params_t;
+
+/* Number of scored windows W_sel (see Geometry).  idx has W_sel * top_k entries per KV head. */
+int lrsa_num_sel_windows(const lrsa_params_t* params, int32_t* w_sel);
+
+/* Workspace sizes in bytes for the three calls (any output pointer may be NULL). */
+int lrsa_workspace_bytes(const lrsa_params_t* params, size_t* score_select, size_t* attn_fwd,
+                         size_t* attn_bwd);
+
+/*
+ * LagKV scoring and selection (Section 3.2, Eq. 4-8 and the selection rule after Eq. 8).
+ * For every batch element, KV head and scored window p: per-channel min and max over the tokens
+ * of window p+1 (Eq. 4, 5) normalise window p (Eq. 6); the per-token standard deviation over
+ * head_dim, soft-maxed over the L tokens of the window (Eq. 7), is computed for K and for V and
+ * the two are added (Eq. 8); the top_k highest-scoring positions are kept.  A channel whose
+ * reference range is zero contributes normalised value 0.  Arithmetic is fp32.
+ *
+ *   K, V   in  : bf16 [B, Hkv, N, d]
+ *   idx    out : int32 [B, Hkv, W_sel, top_k], absolute positions in [0, N), ascending inside
+ *                a window; equal scores keep the lower position.
+ *   score  out : optional (NULL to skip), fp32 [B, Hkv, W_sel, L], the Eq. 8 score.
+ */
+int lrsa_score_select(const lrsa_params_t* params, const void* K, const void* V, int32_t* idx,
+                      float* score, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * LRSA attention forward (Section 3.1, Eq. 3 with the chunked mask of Section 3.2).
+ * Query position t < S attends positions [0, t].  Query t >= S in chunk c = (t-S)/L attends the
+ * sinks, the kept positions idx[b, hkv, w, :] of the first n_c = min(max(c - n_dense_prev, 0),
+ * W_sel) windows, and every position of [S + n_c*L, t].  bf16 tensor-core products, fp32
+ * accumulation and softmax.
+ *
+ *   Q       in  : bf16 [B, Hq, N, d];  K, V in : bf16 [B, Hkv, N, d]
+ *   idx     in  : int32 [B, Hkv, W_sel, top_k]; any set of distinct in-window positions listed
+ *                 ascending per window (normally the output of lrsa_score_select)
+ *   O       out : bf16 [B, Hq, N, d]
+ *   LSE     out : fp32 [B, Hq, N], natural-log sum of exponentials of the scaled scores
+ */
+int lrsa_attn_fwd(const lrsa_params_t* params, const void* Q, const void* K, const void* V,
+                  const int32_t* idx, void* O, float* LSE, void* workspace, size_t workspace_bytes,
+                  void* cuda_stream);
+
+/*
+ * LRSA attention backward: gradient of Eq. 3 with respect to Q, K, V for upstream gradient dO,
+ * the mask (idx) held constant.  P = exp(scale*QK^T - LSE) is recomputed; D = rowsum(dO * O);
+ * dV = P^T dO; dS = P * (dO V^T - D); dQ = scale * dS K; dK = scale * dS^T Q, summed over the
+ * query heads of each KV group; contributions through kept positions land on their original
+ * token positions.  dQ, dK, dV are fully overwritten.
+ *
+ *   O, LSE in : outputs of lrsa_attn_fwd for the same inputs
+ *   dO     in : bf16 [B, Hq, N, d]
+ *   dQ    out : bf16 [B, Hq, N, d];  dK, dV out : bf16 [B, Hkv, N, d]
+ */
+int lrsa_attn_bwd(const lrsa_params_t* params, const void* Q, const void* K, const void* V,
+                  const void* O, const void* dO, const float* LSE, const int32_t* idx, void* dQ,
+                  void* dK, void* dV, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Reads the status word that the last call using `workspace` left there.  Synchronises
+ * `cuda_stream`.  Returns LRSA_OK, LRSA_ERR_TIMEOUT, or LRSA_ERR_CUDA if the copy failed.
+ */
+int lrsa_workspace_status(const void* workspace, void* cuda_stream);
+
+/* Static, human-readable name of a status value. */
+const char* lrsa_status_string(int status);
+
+/* Number of kernels (and memset nodes) the last call on this host thread enqueued. */
+int lrsa_last_launch_count(void);
+
+/*
+ * Validation switch (process-wide): 0 selects the tensor-core attention kernels (default),
+ * 1 the slow CUDA-core kernels kept for cross-checking on the GPU.  Both compute the same
+ * function from the same arguments and workspace.
+ */
+int lrsa_debug_set_impl(int impl);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LRSA_H_ */

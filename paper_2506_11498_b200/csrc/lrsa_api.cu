@@ -1,0 +1,158 @@
+// C ABI entry points: argument validation on the host, workspace layout, kernel dispatch.
+#include <math.h>
+
+#include "lrsa_internal.h"
+
+namespace lrsa {
+
+LaunchCounter& launch_counter() {
+  static thread_local LaunchCounter c;
+  return c;
+}
+
+static int g_impl = 1;  // 0: tensor-core kernels, 1: CUDA-core validation kernels
+
+int make_geom(const lrsa_params_t* p, Geom* g) {
+  if (!p || !g) return LRSA_ERR_INVALID_ARG;
+  if (p->batch < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->seq_len < 1 || p->head_dim < 1 ||
+      p->lag < 1 || p->chunk < 1 || p->top_k < 1 || p->n_sink < 0)
+    return LRSA_ERR_INVALID_ARG;
+  if (p->n_q_heads % p->n_kv_heads != 0) return LRSA_ERR_INVALID_ARG;
+  if (p->top_k > p->lag) return LRSA_ERR_INVALID_ARG;
+  if (p->std_ddof != 0 && p->std_ddof != 1) return LRSA_ERR_INVALID_ARG;
+  if (p->n_dense_prev != 0 && p->n_dense_prev != 1) return LRSA_ERR_INVALID_ARG;
+  if (!(p->softmax_scale >= 0.f) || isinf(p->softmax_scale)) return LRSA_ERR_INVALID_ARG;
+  if (p->head_dim != 64 && p->head_dim != 128) return LRSA_ERR_UNSUPPORTED;
+  if (p->chunk != p->lag) return LRSA_ERR_UNSUPPORTED;
+  if (p->seq_len < p->n_sink) return LRSA_ERR_UNSUPPORTED;
+  if (p->lag > 32767) return LRSA_ERR_UNSUPPORTED;  // packed 16-bit counters in the selection scan
+  if ((long long)p->batch * p->n_q_heads * p->seq_len > 0x7fffffffLL) return LRSA_ERR_UNSUPPORTED;
+  g->B = p->batch; g->Hq = p->n_q_heads; g->Hkv = p->n_kv_heads; g->G = g->Hq / g->Hkv;
+  g->N = p->seq_len; g->d = p->head_dim; g->L = p->lag; g->K = p->top_k; g->S = p->n_sink;
+  g->ndp = p->n_dense_prev; g->ddof = p->std_ddof;
+  g->scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
+  g->W = (g->N - g->S) / g->L;
+  g->T = g->N - g->S - g->W * g->L;
+  g->C = g->W + (g->T > 0 ? 1 : 0);
+  g->Wsel = g->W > 1 ? g->W - 1 : 0;
+  g->Rc = g->S + g->Wsel * g->K;
+  return LRSA_OK;
+}
+
+static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+static size_t fwd_ws_bytes(const Geom& g) { return attn_ref_fwd_ws_bytes(g); }
+static size_t bwd_ws_bytes(const Geom& g) { return attn_ref_bwd_ws_bytes(g); }
+
+}  // namespace lrsa
+
+using namespace lrsa;
+
+extern "C" {
+
+int lrsa_num_sel_windows(const lrsa_params_t* params, int32_t* w_sel) {
+  Geom g;
+  const int rc = make_geom(params, &g);
+  if (rc != LRSA_OK) return rc;
+  if (!w_sel) return LRSA_ERR_INVALID_ARG;
+  *w_sel = g.Wsel;
+  return LRSA_OK;
+}
+
+int lrsa_workspace_bytes(const lrsa_params_t* params, size_t* score_select, size_t* attn_fwd,
+                         size_t* attn_bwd) {
+  Geom g;
+  const int rc = make_geom(params, &g);
+  if (rc != LRSA_OK) return rc;
+  if (score_select) *score_select = score_select_ws_bytes(g);
+  if (attn_fwd) *attn_fwd = fwd_ws_bytes(g);
+  if (attn_bwd) *attn_bwd = bwd_ws_bytes(g);
+  return LRSA_OK;
+}
+
+int lrsa_score_select(const lrsa_params_t* params, const void* K, const void* V, int32_t* idx,
+                      float* score, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  launch_counter().n = 0;
+  Geom g;
+  const int rc = make_geom(params, &g);
+  if (rc != LRSA_OK) return rc;
+  if (!K || !V || !workspace) return LRSA_ERR_INVALID_ARG;
+  if (g.Wsel > 0 && !idx) return LRSA_ERR_INVALID_ARG;
+  if (!aligned(K, 16) || !aligned(V, 16) || !aligned(idx, 4) || !aligned(score, 4) || !aligned(workspace, 256))
+    return LRSA_ERR_INVALID_ARG;
+  if (workspace_bytes < score_select_ws_bytes(g)) return LRSA_ERR_WORKSPACE_TOO_SMALL;
+  return launch_score_select(g, static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(V),
+                             idx, score, workspace, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int lrsa_attn_fwd(const lrsa_params_t* params, const void* Q, const void* K, const void* V,
+                  const int32_t* idx, void* O, float* LSE, void* workspace, size_t workspace_bytes,
+                  void* cuda_stream) {
+  launch_counter().n = 0;
+  Geom g;
+  const int rc = make_geom(params, &g);
+  if (rc != LRSA_OK) return rc;
+  if (!Q || !K || !V || !O || !LSE || !workspace) return LRSA_ERR_INVALID_ARG;
+  if (g.Wsel > 0 && !idx) return LRSA_ERR_INVALID_ARG;
+  if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(LSE, 16) ||
+      !aligned(idx, 4) || !aligned(workspace, 256))
+    return LRSA_ERR_INVALID_ARG;
+  if (workspace_bytes < fwd_ws_bytes(g)) return LRSA_ERR_WORKSPACE_TOO_SMALL;
+  auto st = static_cast<cudaStream_t>(cuda_stream);
+  return launch_attn_ref_fwd(g, static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
+                             static_cast<const __nv_bfloat16*>(V), idx, static_cast<__nv_bfloat16*>(O), LSE,
+                             workspace, st);
+}
+
+int lrsa_attn_bwd(const lrsa_params_t* params, const void* Q, const void* K, const void* V,
+                  const void* O, const void* dO, const float* LSE, const int32_t* idx, void* dQ,
+                  void* dK, void* dV, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  launch_counter().n = 0;
+  Geom g;
+  const int rc = make_geom(params, &g);
+  if (rc != LRSA_OK) return rc;
+  if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV || !workspace) return LRSA_ERR_INVALID_ARG;
+  if (g.Wsel > 0 && !idx) return LRSA_ERR_INVALID_ARG;
+  const void* ptrs[] = {Q, K, V, O, dO, LSE, dQ, dK, dV};
+  for (const void* p : ptrs)
+    if (!aligned(p, 16)) return LRSA_ERR_INVALID_ARG;
+  if (!aligned(idx, 4) || !aligned(workspace, 256)) return LRSA_ERR_INVALID_ARG;
+  if (workspace_bytes < bwd_ws_bytes(g)) return LRSA_ERR_WORKSPACE_TOO_SMALL;
+  auto st = static_cast<cudaStream_t>(cuda_stream);
+  auto bf = [](const void* p) { return static_cast<const __nv_bfloat16*>(p); };
+  return launch_attn_ref_bwd(g, bf(Q), bf(K), bf(V), bf(O), bf(dO), LSE, idx,
+                             static_cast<__nv_bfloat16*>(dQ), static_cast<__nv_bfloat16*>(dK),
+                             static_cast<__nv_bfloat16*>(dV), workspace, st);
+}
+
+int lrsa_workspace_status(const void* workspace, void* cuda_stream) {
+  if (!workspace) return LRSA_ERR_INVALID_ARG;
+  int status = 0;
+  auto st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(&status, workspace, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return LRSA_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return LRSA_ERR_CUDA;
+  return status == 0 ? LRSA_OK : LRSA_ERR_TIMEOUT;
+}
+
+const char* lrsa_status_string(int status) {
+  switch (status) {
+    case LRSA_OK: return "ok";
+    case LRSA_ERR_INVALID_ARG: return "invalid argument";
+    case LRSA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case LRSA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case LRSA_ERR_CUDA: return "CUDA runtime error";
+    case LRSA_ERR_TIMEOUT: return "bounded device-side wait expired";
+    default: return "unknown status";
+  }
+}
+
+int lrsa_last_launch_count(void) { return launch_counter().n; }
+
+int lrsa_debug_set_impl(int impl) {
+  if (impl != 0 && impl != 1) return LRSA_ERR_INVALID_ARG;
+  g_impl = impl;
+  return LRSA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,78 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/lrsa.h"
+
+namespace lrsa {
+
+// Problem geometry derived from lrsa_params_t (Section 3.2: sink of size S, windows of lag L).
+struct Geom {
+  int B, Hq, Hkv, G, N, d, L, K, S, ndp, ddof;
+  float scale;
+  int W;     // full windows
+  int T;     // tail tokens
+  int C;     // query chunks = W + [T > 0]
+  int Wsel;  // scored windows = max(W - 1, 0)
+  int Rc;    // rows of the compact (sinks + kept) K/V buffer per KV head = S + Wsel*K
+};
+
+// Validates `p` and fills `g`. Returns an lrsa_status.
+int make_geom(const lrsa_params_t* p, Geom* g);
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Workspace header (first 256 bytes of every workspace).
+struct WsHeader {
+  int status;   // lrsa_status written by kernels (0 or LRSA_ERR_TIMEOUT)
+  int ticket;   // dynamic work counter of the scoring kernel
+  int pad[62];
+};
+static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
+
+// Number of leading windows that query chunk c sees only through their kept tokens.
+__host__ __device__ inline int n_hist_windows(int c, int ndp, int Wsel) {
+  int n = c - ndp;
+  if (n < 0) n = 0;
+  return n < Wsel ? n : Wsel;
+}
+
+// First chunk that sees window w compressed (C if none): smallest c with n_hist_windows(c) > w.
+__host__ __device__ inline int first_compressed_chunk(int w, int ndp, int Wsel, int C) {
+  if (w >= Wsel) return C;
+  int c = w + 1 + ndp;
+  return c < C ? c : C;
+}
+
+struct LaunchCounter {
+  int n = 0;
+};
+LaunchCounter& launch_counter();
+
+// score_select.cu
+size_t score_select_ws_bytes(const Geom& g);
+int launch_score_select(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat16* V, int32_t* idx,
+                        float* score, void* ws, cudaStream_t st);
+
+// attn_ref.cu : CUDA-core reference kernels (one warp per row), used for validation.
+size_t attn_ref_fwd_ws_bytes(const Geom& g);
+size_t attn_ref_bwd_ws_bytes(const Geom& g);
+int launch_attn_ref_fwd(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
+                        const __nv_bfloat16* V, const int32_t* idx, __nv_bfloat16* O, float* LSE,
+                        void* ws, cudaStream_t st);
+int launch_attn_ref_bwd(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
+                        const __nv_bfloat16* V, const __nv_bfloat16* O, const __nv_bfloat16* dO,
+                        const float* LSE, const int32_t* idx, __nv_bfloat16* dQ, __nv_bfloat16* dK,
+                        __nv_bfloat16* dV, void* ws, cudaStream_t st);
+
+#define LRSA_CUDA_CHECK(expr)                                 \
+  do {                                                        \
+    cudaError_t _e = (expr);                                  \
+    if (_e != cudaSuccess) return (int)LRSA_ERR_CUDA;         \
+  } while (0)
+
+}  // namespace lrsa

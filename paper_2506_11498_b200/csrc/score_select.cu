@@ -1,0 +1,414 @@
+// LagKV scoring and top-K selection (Section 3.2, Eq. 4-8 and the selection rule after Eq. 8).
+//
+// One launch streams K and V exactly once.  The work unit is a slice of TOK tokens of one lag
+// window of one (batch, KV head); a CTA takes units from a ticket counter in DESCENDING window
+// order and keeps its slice of K and V in registers for both phases:
+//   phase 1  per-channel min/max of the slice (packed bf16x2 compares, exact), folded into the
+//            window's statistics in global memory with order-preserving integer atomics, then
+//            a release-increment of the window's `ready` counter            (Eq. 4, Eq. 5)
+//   phase 2  wait (bounded) until the FOLLOWING window's statistics are complete, normalise
+//            the slice held in registers (Eq. 6), per-token standard deviation over head_dim
+//            (Eq. 7, inner part), written to a small fp32 scratch
+//   select   the CTA that finishes a window last soft-maxes the window's K and V spreads
+//            (Eq. 7), adds them (Eq. 8), radix-selects the top_k scores and emits the kept
+//            positions in ascending order.
+// A unit of window w waits only on units of window w+1, all of which hold smaller tickets, were
+// therefore picked up by CTAs that already run, and publish before they wait on anything: the
+// wait always ends, whatever the number of resident CTAs.  It is bounded all the same.
+#include "lrsa_internal.h"
+
+namespace lrsa {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kSteps = 4;  // 16-byte row chunks of K (and of V) each thread keeps in registers
+
+struct ScoreArgs {
+  const __nv_bfloat16* K;
+  const __nv_bfloat16* V;
+  int32_t* idx;
+  float* score;   // optional
+  WsHeader* hdr;
+  int* ready;     // [BH, W]     slices of window w whose min/max are folded in
+  int* done;      // [BH, Wsel]  slices of window w whose spreads are written
+  uint32_t* mm;   // [BH, W, 2 (K,V), 2 (min,max), d] order-preserving keys, zero = identity
+  float* spread;  // [BH, Wsel, 2 (K,V), L]
+  int BH, N, L, Kk, S, W, Wsel, n_slices, ddof;
+  int spin_limit;
+};
+
+// fp32 bits -> uint32 whose unsigned order is the float order (and back).
+__device__ __forceinline__ uint32_t order_key(float f) {
+  uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_to_float(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k ^ 0x80000000u) : ~k);
+}
+
+__device__ __forceinline__ uint32_t bmin2(uint32_t a, uint32_t b) {
+  __nv_bfloat162 r = __hmin2(*reinterpret_cast<__nv_bfloat162*>(&a), *reinterpret_cast<__nv_bfloat162*>(&b));
+  return *reinterpret_cast<uint32_t*>(&r);
+}
+__device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b) {
+  __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162*>(&a), *reinterpret_cast<__nv_bfloat162*>(&b));
+  return *reinterpret_cast<uint32_t*>(&r);
+}
+__device__ __forceinline__ float bf_lo(uint32_t p) { return __uint_as_float(p << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t p) { return __uint_as_float(p & 0xffff0000u); }
+
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Top-K of the window by the last CTA to finish it.  smem: sk[L], sv[L] floats, then scratch.
+__device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* smem) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, L = a.L;
+  float* sk = reinterpret_cast<float*>(smem);
+  float* sv = sk + L;
+  uint32_t* hist = reinterpret_cast<uint32_t*>(sv + L);  // 256 bins
+  float* red = reinterpret_cast<float*>(hist + 256);     // 32 floats
+  int* ibuf = reinterpret_cast<int*>(red + 32);          // 16 ints
+  const float* gk = a.spread + ((size_t)(bh * a.Wsel + w) * 2 + 0) * L;
+  const float* gv = gk + L;
+
+  // Eq. 7: softmax over the L tokens of the window, for K and for V
+  float mk = -INFINITY, mv = -INFINITY;
+  for (int i = tid; i < L; i += kThreads) {
+    const float x = __ldcg(gk + i), y = __ldcg(gv + i);
+    sk[i] = x; sv[i] = y;
+    mk = fmaxf(mk, x); mv = fmaxf(mv, y);
+  }
+  mk = warp_max(mk); mv = warp_max(mv);
+  if (lane == 0) { red[warp] = mk; red[8 + warp] = mv; }
+  __syncthreads();
+  mk = red[0]; mv = red[8];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) { mk = fmaxf(mk, red[i]); mv = fmaxf(mv, red[8 + i]); }
+  __syncthreads();
+  float ek = 0.f, ev = 0.f;
+  for (int i = tid; i < L; i += kThreads) {
+    const float x = expf(sk[i] - mk), y = expf(sv[i] - mv);
+    sk[i] = x; sv[i] = y;
+    ek += x; ev += y;
+  }
+  ek = warp_sum(ek); ev = warp_sum(ev);
+  if (lane == 0) { red[warp] = ek; red[8 + warp] = ev; }
+  __syncthreads();
+  ek = 0.f; ev = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { ek += red[i]; ev += red[8 + i]; }
+  // Eq. 8
+  float* gs = a.score ? a.score + (size_t)(bh * a.Wsel + w) * L : nullptr;
+  for (int i = tid; i < L; i += kThreads) {
+    const float s = sk[i] / ek + sv[i] / ev;
+    sk[i] = s;
+    if (gs) gs[i] = s;
+  }
+  __syncthreads();
+
+  // radix select of the K-th largest score; scores are positive, so bit order = value order
+  const uint32_t* key = reinterpret_cast<const uint32_t*>(sk);
+  uint32_t prefix = 0, mask = 0;
+  int remaining = a.Kk;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    hist[tid] = 0;
+    __syncthreads();
+    for (int i = tid; i < L; i += kThreads) {
+      const uint32_t k = key[i];
+      if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (warp == 0) {
+      // lane l owns bins 255-8l ... 248-8l, highest first
+      uint32_t c[8], tot = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { c[j] = hist[255 - 8 * lane - j]; tot += c[j]; }
+      uint32_t incl = tot;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+      }
+      uint32_t above = incl - tot;  // elements in bins above this lane's
+      if (above < (uint32_t)remaining && (uint32_t)remaining <= incl) {
+        int j = 0;
+        while (above + c[j] < (uint32_t)remaining) { above += c[j]; ++j; }
+        ibuf[0] = 255 - 8 * lane - j;
+        ibuf[1] = remaining - (int)above;
+      }
+    }
+    __syncthreads();
+    prefix |= (uint32_t)ibuf[0] << shift;
+    mask |= 255u << shift;
+    remaining = ibuf[1];
+    __syncthreads();
+  }
+  const uint32_t kth = prefix;    // K-th largest key
+  const int need_eq = remaining;  // how many keys equal to it are kept (lowest positions first)
+
+  // emit kept positions in ascending order
+  int32_t* out = a.idx + (size_t)(bh * a.Wsel + w) * a.Kk;
+  int base_gt = 0, base_eq = 0;
+  int* wtot = ibuf;  // 8 warp totals
+  for (int i0 = 0; i0 < L; i0 += kThreads) {
+    const int i = i0 + tid;
+    const uint32_t k = i < L ? key[i] : 0u;
+    const int gt = (i < L && k > kth) ? 1 : 0, eq = (i < L && k == kth) ? 1 : 0;
+    const int packed = gt | (eq << 16);
+    int incl = packed;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    if (lane == 31) wtot[warp] = incl;
+    __syncthreads();
+    int excl = incl - packed, all = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int t = wtot[j];
+      if (j < warp) excl += t;
+      all += t;
+    }
+    const int gt_before = base_gt + (excl & 0xffff), eq_before = base_eq + (excl >> 16);
+    if (gt || (eq && eq_before < need_eq))
+      out[gt_before + min(eq_before, need_eq)] = a.S + w * L + i;
+    base_gt += all & 0xffff;
+    base_eq += all >> 16;
+    __syncthreads();
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads) score_select_kernel(const ScoreArgs a) {
+  constexpr int LPR = D / 8;              // lanes per token row, 16 bytes each
+  constexpr int RPS = kThreads / LPR;     // rows per step
+  constexpr int TOK = kSteps * RPS;       // tokens per unit
+  extern __shared__ __align__(16) unsigned char smem[];
+  __shared__ int s_ticket, s_flag;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) { s_ticket = atomicAdd(&a.hdr->ticket, 1); s_flag = 0; }
+  __syncthreads();
+  const int per_w = a.BH * a.n_slices;
+  const int w = a.W - 1 - s_ticket / per_w;   // descending windows
+  const int r = s_ticket % per_w;
+  const int bh = r / a.n_slices, slice = r % a.n_slices;
+  const int chunk = tid % LPR, row = tid / LPR;
+
+  // the slice of K and of V, held in registers for both phases
+  uint4 kq[kSteps], vq[kSteps];
+  bool valid[kSteps];
+  const size_t row0 = (size_t)bh * a.N + a.S + (size_t)w * a.L;
+#pragma unroll
+  for (int s = 0; s < kSteps; ++s) {
+    const int i = slice * TOK + s * RPS + row;
+    valid[s] = i < a.L;
+    if (valid[s]) {
+      const size_t off = (row0 + i) * D + chunk * 8;
+      kq[s] = __ldcs(reinterpret_cast<const uint4*>(a.K + off));
+      vq[s] = __ldcs(reinterpret_cast<const uint4*>(a.V + off));
+    } else {
+      kq[s] = make_uint4(0, 0, 0, 0);
+      vq[s] = make_uint4(0, 0, 0, 0);
+    }
+  }
+
+  // ---- phase 1: Eq. 4, Eq. 5 (window 0 is never a reference) ----
+  if (w >= 1) {
+    const uint32_t PINF = 0x7F807F80u, NINF = 0xFF80FF80u;
+    uint32_t st[2][2][4];  // [K,V][min,max][4 bf16 pairs]
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { st[0][0][j] = st[1][0][j] = PINF; st[0][1][j] = st[1][1][j] = NINF; }
+#pragma unroll
+    for (int s = 0; s < kSteps; ++s) {
+      if (!valid[s]) continue;
+      const uint32_t kk[4] = {kq[s].x, kq[s].y, kq[s].z, kq[s].w};
+      const uint32_t vv[4] = {vq[s].x, vq[s].y, vq[s].z, vq[s].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        st[0][0][j] = bmin2(st[0][0][j], kk[j]); st[0][1][j] = bmax2(st[0][1][j], kk[j]);
+        st[1][0][j] = bmin2(st[1][0][j], vv[j]); st[1][1][j] = bmax2(st[1][1][j], vv[j]);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o >= LPR; o >>= 1)
+#pragma unroll
+      for (int z = 0; z < 2; ++z)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          st[z][0][j] = bmin2(st[z][0][j], __shfl_xor_sync(0xffffffffu, st[z][0][j], o));
+          st[z][1][j] = bmax2(st[z][1][j], __shfl_xor_sync(0xffffffffu, st[z][1][j], o));
+        }
+    // cross-warp: smem [warp][z*2+stat][D] bf16
+    __nv_bfloat16* sm = reinterpret_cast<__nv_bfloat16*>(smem);
+    if (lane < LPR) {
+#pragma unroll
+      for (int z = 0; z < 2; ++z)
+#pragma unroll
+        for (int m = 0; m < 2; ++m)
+          *reinterpret_cast<uint4*>(sm + ((warp * 4 + z * 2 + m) * D + lane * 8)) =
+              make_uint4(st[z][m][0], st[z][m][1], st[z][m][2], st[z][m][3]);
+    }
+    __syncthreads();
+    uint32_t* mm = a.mm + (size_t)(bh * a.W + w) * 4 * D;
+    for (int v = tid; v < 4 * D; v += kThreads) {
+      const int zs = v / D, ch = v % D;
+      const bool is_max = zs & 1;
+      float acc = __bfloat162float(sm[zs * D + ch]);
+#pragma unroll
+      for (int ww = 1; ww < kThreads / 32; ++ww) {
+        const float x = __bfloat162float(sm[(ww * 4 + zs) * D + ch]);
+        acc = is_max ? fmaxf(acc, x) : fminf(acc, x);
+      }
+      const uint32_t k = order_key(acc);
+      atomicMax(mm + v, is_max ? k : ~k);
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) atomicAdd(a.ready + bh * a.W + w, 1);
+  }
+  if (w >= a.Wsel) return;  // the last full window is a reference only
+
+  // ---- phase 2: Eq. 6 and the per-token Std of Eq. 7 ----
+  if (tid == 0) {
+    const int* flag = a.ready + bh * a.W + w + 1;
+    int it = 0;
+    while (ld_acquire(flag) < a.n_slices) {
+      if (++it > a.spin_limit) { s_flag = 1; atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT); break; }
+      __nanosleep(64);
+    }
+  }
+  __syncthreads();
+  if (s_flag) return;
+  __threadfence();
+
+  const uint32_t* mm = a.mm + (size_t)(bh * a.W + w + 1) * 4 * D;
+  const float inv_dof = 1.0f / (float)(D - a.ddof);
+#pragma unroll
+  for (int z = 0; z < 2; ++z) {
+    // z' = x*sa + sb = zbar - 1/2; a channel with zero range has zbar = 0
+    float sa[8], sb[8];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const uint4 kmn = __ldcg(reinterpret_cast<const uint4*>(mm + (z * 2 + 0) * D + chunk * 8 + h * 4));
+      const uint4 kmx = __ldcg(reinterpret_cast<const uint4*>(mm + (z * 2 + 1) * D + chunk * 8 + h * 4));
+      const uint32_t a_mn[4] = {kmn.x, kmn.y, kmn.z, kmn.w}, a_mx[4] = {kmx.x, kmx.y, kmx.z, kmx.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float mn = key_to_float(~a_mn[j]), mx = key_to_float(a_mx[j]);
+        const float range = mx - mn;
+        const float inv = range > 0.f ? 1.0f / range : 0.f;
+        sa[h * 4 + j] = inv;
+        sb[h * 4 + j] = range > 0.f ? -(0.5f * (mn + mx)) * inv : -0.5f;
+      }
+    }
+    float* out = a.spread + ((size_t)(bh * a.Wsel + w) * 2 + z) * a.L;
+#pragma unroll
+    for (int s = 0; s < kSteps; ++s) {
+      const uint4 q = z == 0 ? kq[s] : vq[s];
+      const uint32_t pk[4] = {q.x, q.y, q.z, q.w};
+      float sum = 0.f, sq = 0.f;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float z0 = fmaf(bf_lo(pk[j]), sa[2 * j], sb[2 * j]);
+        const float z1 = fmaf(bf_hi(pk[j]), sa[2 * j + 1], sb[2 * j + 1]);
+        sum += z0 + z1;
+        sq = fmaf(z0, z0, sq);
+        sq = fmaf(z1, z1, sq);
+      }
+#pragma unroll
+      for (int o = LPR / 2; o > 0; o >>= 1) {
+        sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        sq += __shfl_xor_sync(0xffffffffu, sq, o);
+      }
+      if (chunk == 0 && valid[s]) {
+        const float var = (sq - sum * sum * (1.0f / D)) * inv_dof;
+        out[slice * TOK + s * RPS + row] = sqrtf(fmaxf(var, 0.f));
+      }
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_flag = (atomicAdd(a.done + bh * a.Wsel + w, 1) == a.n_slices - 1) ? 2 : 0;
+  __syncthreads();
+  if (s_flag != 2) return;
+  __threadfence();
+  select_window(a, bh, w, smem);
+}
+
+template <int D>
+constexpr int tok_per_unit() { return kSteps * (kThreads / (D / 8)); }
+
+size_t select_smem_bytes(int L, int d) {
+  const size_t phase1 = (size_t)(kThreads / 32) * 4 * d * sizeof(__nv_bfloat16);
+  const size_t sel = (size_t)2 * L * sizeof(float) + 256 * 4 + 32 * 4 + 16 * 4;
+  return phase1 > sel ? phase1 : sel;
+}
+
+struct ScoreWs {
+  size_t ready, done, mm, zero_bytes, spread, total;
+};
+ScoreWs score_ws_layout(const Geom& g) {
+  ScoreWs w;
+  const size_t BH = (size_t)g.B * g.Hkv;
+  size_t off = sizeof(WsHeader);
+  w.ready = off; off += align_up(BH * g.W * sizeof(int), 16);
+  w.done = off;  off += align_up(BH * g.Wsel * sizeof(int), 16);
+  w.mm = off;    off += align_up(BH * g.W * 4 * g.d * sizeof(uint32_t), 256);
+  w.zero_bytes = off;   // everything up to here is cleared before the launch
+  w.spread = off; off += align_up(BH * g.Wsel * 2 * g.L * sizeof(float), 256);
+  w.total = off;
+  return w;
+}
+
+}  // namespace
+
+size_t score_select_ws_bytes(const Geom& g) { return score_ws_layout(g).total; }
+
+int launch_score_select(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat16* V, int32_t* idx,
+                        float* score, void* ws, cudaStream_t st) {
+  if (g.Wsel == 0) return LRSA_OK;  // nothing is scored
+  const ScoreWs lay = score_ws_layout(g);
+  unsigned char* base = static_cast<unsigned char*>(ws);
+  LRSA_CUDA_CHECK(cudaMemsetAsync(base, 0, lay.zero_bytes, st));
+  launch_counter().n++;
+  ScoreArgs a;
+  a.K = K; a.V = V; a.idx = idx; a.score = score;
+  a.hdr = reinterpret_cast<WsHeader*>(base);
+  a.ready = reinterpret_cast<int*>(base + lay.ready);
+  a.done = reinterpret_cast<int*>(base + lay.done);
+  a.mm = reinterpret_cast<uint32_t*>(base + lay.mm);
+  a.spread = reinterpret_cast<float*>(base + lay.spread);
+  a.BH = g.B * g.Hkv; a.N = g.N; a.L = g.L; a.Kk = g.K; a.S = g.S; a.W = g.W; a.Wsel = g.Wsel;
+  a.ddof = g.ddof;
+  a.spin_limit = 1 << 21;
+  const int tok = g.d == 128 ? tok_per_unit<128>() : tok_per_unit<64>();
+  a.n_slices = (g.L + tok - 1) / tok;
+  const size_t smem = select_smem_bytes(g.L, g.d);
+  if (smem > 200 * 1024) return LRSA_ERR_UNSUPPORTED;
+  const long long units = (long long)a.BH * g.W * a.n_slices;
+  if (units > 0x7fffffffLL) return LRSA_ERR_UNSUPPORTED;
+  auto kern = g.d == 128 ? score_select_kernel<128> : score_select_kernel<64>;
+  LRSA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kern<<<(unsigned)units, kThreads, smem, st>>>(a);
+  LRSA_CUDA_CHECK(cudaGetLastError());
+  launch_counter().n++;
+  return LRSA_OK;
+}
+
+}  // namespace lrsa
