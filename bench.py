@@ -1,0 +1,367 @@
+#!/usr/bin/env python
+"""Benchmark of the LRSA hot path: score/select + attention forward + backward on one layer.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A step is one pass of the whole path (lrsa_score_select, lrsa_attn_fwd, lrsa_attn_bwd) over one
+batch of seeded synthetic bf16 tensors shaped like a 32K-token post-training sequence of a
+7B-class GQA layer.  Prints ONE JSON line (rank 0).  `--impl reference` times the fp64 CPU checker
+under oracle/ on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "lrsa_fwd_bwd_effective_tflops"
+UNIT = "TFLOP/s"
+
+
+def geometry(w, ndp=1):
+    W = (w.N - w.S) // w.L
+    T = w.N - w.S - W * w.L
+    C = W + (1 if T > 0 else 0)
+    return W, T, C, max(W - 1, 0)
+
+
+def count_pairs(w, ndp=1) -> int:
+    """Unmasked (query, key) pairs per query head: sinks causal among themselves; a query of chunk c
+    sees S sinks, K kept keys from each compressed window, the uncompressed windows before it, and
+    its own chunk causally."""
+    W, T, C, Wsel = geometry(w, ndp)
+    pairs = w.S * (w.S + 1) // 2
+    for c in range(C):
+        n_c = w.L if c < W else T
+        nh = min(max(c - ndp, 0), Wsel)
+        pairs += n_c * (w.S + nh * w.K + (c - nh) * w.L) + n_c * (n_c + 1) // 2
+    return pairs
+
+
+def flops(w, ndp=1):
+    """Effective FLOPs: 4*d per pair forward (QK^T, PV), 10*d backward (five products)."""
+    p = count_pairs(w, ndp) * w.Hq * w.B
+    return 4 * w.d * p, 10 * w.d * p
+
+
+def kv_bytes(w):
+    Wsel = geometry(w)[3]
+    return 2 * w.B * w.Hkv * w.N * w.d * 2 + w.B * w.Hkv * Wsel * w.K * 4
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        m = json.load(open(path))
+        return {"hbm_gbs": m["hbm_gbs"], "bf16_tflops": m["bf16_tflops"],
+                "bf16_tflops_sustained": m.get("bf16_tflops_sustained", m["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            busy = [x for x in sm if x > 0]
+            out["sm_mhz"] = statistics.median(busy) if busy else None
+            out["sm_max_mhz"] = max(mx)
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def oracle_sample(w, n_chunks=3, host=None):
+    """Times the fp64 CPU checker, as it stands, on a bounded sample of workload `w`: the first
+    S + n_chunks*L tokens of KV-head group 0 of batch element 0 (all of its query heads).  Attention
+    is causal, so this prefix is a self-contained part of the workload: its outputs equal the
+    full run's.  Returns the seconds of each leg and the effective FLOPs the sample covers."""
+    import numpy as np
+    from oracle import lrsa_oracle as orc
+    from paper_2506_11498_b200 import workloads
+    host = host if host is not None else workloads.generate(w)
+    G = w.Hq // w.Hkv
+    n = min(w.N, w.S + n_chunks * w.L)
+    sub = w.with_(name=w.name + "_prefix", B=1, Hq=G, Hkv=1, N=n)
+    bits = {k: np.ascontiguousarray(orc.bf16_bits(v)[:1, :(G if k in ("Q", "dO") else 1), :n]) for k, v in host.items()}
+    op = orc.OracleParams(sub.B, sub.Hq, sub.Hkv, sub.N, sub.d, sub.L, sub.K, sub.S)
+    t0 = time.perf_counter()
+    idx, _ = orc.score_select(op, bits["K"], bits["V"])
+    t_score = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    orc.attn_fwd(op, bits["Q"], bits["K"], bits["V"], idx)
+    t_fwd = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    orc.attn_bwd(op, bits["Q"], bits["K"], bits["V"], bits["dO"], idx)
+    t_bwd = time.perf_counter() - t0
+    f_fwd, f_bwd = flops(sub)
+    total = t_score + t_fwd + t_bwd
+    return {"t_score": t_score, "t_fwd": t_fwd, "t_bwd": t_bwd, "seconds": total,
+            "tflops": (f_fwd + f_bwd) / total / 1e12, "tokens_per_s": n / total / w.Hkv,
+            "cores": orc.num_threads(),
+            "sample": f"first {n} tokens (sinks + {n_chunks} chunks) of KV group 0 of batch 0 of {w.name}: "
+                      f"{G} query heads, full score/select + forward + backward, {total:.1f} s of CPU work"}
+
+
+def run_reference(args, w):
+    """Reference arm: the CPU checker on host cores, each step a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    f_fwd, f_bwd = flops(w)
+    vals = []
+    from paper_2506_11498_b200 import workloads
+    host = workloads.generate(w)
+    for i in range(args.warmup + args.steps):
+        s = oracle_sample(w, n_chunks=2, host=host)
+        if i >= args.warmup:
+            vals.append(s)
+    value = statistics.mean(v["tflops"] for v in vals)
+    proj = (f_fwd + f_bwd) / (value * 1e12)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": proj * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "N": w.N, "Hq": w.Hq, "Hkv": w.Hkv, "d": w.d, "L": w.L,
+                   "K": w.K, "S": w.S, "note": "each step is a bounded sample; ms_per_step is the whole-workload time at the sample's rate"},
+        "tokens_per_s": w.B * w.N / proj,
+        "sample_seconds_per_step": statistics.mean(v["seconds"] for v in vals),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": vals[-1]["cores"], "kind": "oracle",
+                         "sample": vals[-1]["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2_32k_gqa7_d128")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    from paper_2506_11498_b200 import workloads
+    w = workloads.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    from paper_2506_11498_b200 import lrsa
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    # weak scaling: every rank runs its own sequence (independent problems, no data-path collective)
+    wl = w.with_(seed=w.seed + 1000 * rank)
+    lrsa.lib()
+    p = lrsa.Params.from_workload(wl)
+    host = {k: v.pin_memory() for k, v in workloads.generate(wl).items()}
+    dev = {k: v.cuda(non_blocking=True) for k, v in host.items()}
+    ws_sizes = lrsa.lrsa_workspace_bytes(p)
+    ws = [lrsa.new_workspace(n) for n in ws_sizes]
+    wsel = lrsa.lrsa_num_sel_windows(p)
+    idx = torch.empty((wl.B, wl.Hkv, wsel, wl.K), dtype=torch.int32, device="cuda")
+    O = torch.empty_like(dev["Q"]); LSE = torch.empty(dev["Q"].shape[:3], dtype=torch.float32, device="cuda")
+    dQ = torch.empty_like(dev["Q"]); dK = torch.empty_like(dev["K"]); dV = torch.empty_like(dev["V"])
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # > 126 MB L2
+    stream = torch.cuda.current_stream()
+    launches = [0]
+
+    def step(timers=None):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if timers is not None else None
+        if ev: ev[0].record(stream)
+        lrsa.lrsa_score_select(p, dev["K"], dev["V"], idx=idx, workspace=ws[0])
+        n = lrsa.lrsa_last_launch_count()
+        if ev: ev[1].record(stream)
+        lrsa.lrsa_attn_fwd(p, dev["Q"], dev["K"], dev["V"], idx, O=O, LSE=LSE, workspace=ws[1])
+        n += lrsa.lrsa_last_launch_count()
+        if ev: ev[2].record(stream)
+        lrsa.lrsa_attn_bwd(p, dev["Q"], dev["K"], dev["V"], O, dev["dO"], LSE, idx, dQ=dQ, dK=dK, dV=dV,
+                           workspace=ws[2])
+        n += lrsa.lrsa_last_launch_count()
+        if ev:
+            ev[3].record(stream)
+            timers.append(ev)
+        launches[0] = n
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        flush.zero_()
+        step()
+    barrier()
+    for i, s in enumerate(ws):
+        st = lrsa.lrsa_workspace_status(s)
+        if st != 0:
+            raise SystemExit(f"workspace {i} reports {lrsa.STATUS.get(st, st)}")
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    timers = []
+    barrier()
+    for _ in range(args.steps):
+        flush.zero_()              # L2 flush between timed iterations (outside the per-step events)
+        step(timers)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    t_score = [e[0].elapsed_time(e[1]) for e in timers]
+    t_fwd = [e[1].elapsed_time(e[2]) for e in timers]
+    t_bwd = [e[2].elapsed_time(e[3]) for e in timers]
+    t_step = [e[0].elapsed_time(e[3]) for e in timers]
+    total_ms = sum(t_step)
+    if dist is not None:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+
+    # end to end through the C ABI with HOST buffers: H2D of Q,K,V,dO from pinned memory and D2H
+    # of O,dQ,dK,dV inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        outs_host = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in
+                     (("O", O), ("dQ", dQ), ("dK", dK), ("dV", dV))}
+        h2d = sum(v.numel() * v.element_size() for v in host.values())
+        d2h = sum(v.numel() * v.element_size() for v in outs_host.values())
+
+        def e2e_step():
+            for k in dev:
+                dev[k].copy_(host[k], non_blocking=True)
+            step()
+            for k, t in (("O", O), ("dQ", dQ), ("dK", dK), ("dV", dV)):
+                outs_host[k].copy_(t, non_blocking=True)
+
+        e2e_step(); barrier()
+        n_e2e = max(2, min(args.steps, 5))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for _ in range(n_e2e):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / n_e2e
+        if dist is not None:
+            t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        f_fwd, f_bwd = flops(wl)
+        e2e = {"value": world * (f_fwd + f_bwd) / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+               "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    f_fwd, f_bwd = flops(wl)
+    peaks = measured_peaks()
+    med = statistics.median
+    bwd_s, fwd_s, score_s = med(t_bwd) * 1e-3, med(t_fwd) * 1e-3, med(t_score) * 1e-3
+    # the kernel is timed inside a long step under the power cap: sustained bf16 peak
+    peak_tf = peaks["bf16_tflops_sustained"]
+    achieved = f_bwd / bwd_s / 1e12
+    line = {
+        "metric": METRIC, "value": world * (f_fwd + f_bwd) / (ms_per_step * 1e-3) / 1e12, "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "B": wl.B, "N": wl.N, "Hq": wl.Hq, "Hkv": wl.Hkv, "d": wl.d,
+                   "L": wl.L, "K": wl.K, "S": wl.S, "values": wl.values,
+                   "l2": "256 MB buffer written between timed steps (outside the per-step events)",
+                   "parallelism": f"replicas x{world} (independent sequences, no collective)"},
+        "tokens_per_s": world * wl.B * wl.N / (ms_per_step * 1e-3),
+        "pct_of_bf16_peak": {"measured_sustained": 100 * (f_fwd + f_bwd) / (ms_per_step * 1e-3) / 1e12 / peak_tf,
+                             "measured_burst": 100 * (f_fwd + f_bwd) / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                             "nominal_2250": 100 * (f_fwd + f_bwd) / (ms_per_step * 1e-3) / 1e12 / 2250.0},
+        "stages_ms": {"score_select": med(t_score), "attn_fwd": med(t_fwd), "attn_bwd": med(t_bwd),
+                      "score_select_min": min(t_score), "attn_fwd_min": min(t_fwd), "attn_bwd_min": min(t_bwd)},
+        "stage_rates": {"fwd_tflops": f_fwd / fwd_s / 1e12, "bwd_tflops": f_bwd / bwd_s / 1e12,
+                        "score_select_gbs": kv_bytes(wl) / score_s / 1e9,
+                        "score_select_frac_of_hbm": kv_bytes(wl) / score_s / 1e9 / peaks["hbm_gbs"]},
+        "roofline": {"kernel": "lrsa_attn_bwd", "bound": "tensor", "achieved": achieved, "peak": peak_tf,
+                     "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": None,
+                     "peak_source": f"{peaks['source']} sustained bf16"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches[0] * args.steps,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        s = oracle_sample(w, n_chunks=3, host={k: v for k, v in host.items()} if wl.seed == w.seed else None)
+        line["cpu_baseline"] = {"value": s["tflops"], "unit": UNIT, "cores": s["cores"], "kind": "oracle",
+                                "sample": s["sample"]}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
