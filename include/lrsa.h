@@ -88,6 +88,31 @@ int lrsa_score_select(const lrsa_params_t* params, const void* K, const void* V,
                       float* score, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Same computation and outputs as lrsa_score_select, for callers that can neither supply a
+ * workspace nor let the library allocate one (the paper has no counterpart; this is a packaging
+ * variant).  Typical case: a plugin running inside a process whose caching allocator already owns
+ * all device memory, or a loop that must not enter cudaMalloc/cudaFree because of their device-wide
+ * synchronisation.  The scratch is a fixed array of LRSA_STATIC_SCRATCH_BYTES inside the library's
+ * device image: every GPU that loads the library holds that much memory until the process exits.
+ *
+ *   - Allocates nothing: no cudaMalloc/cudaFree, no allocating library routine.  The caller still
+ *     passes K, V (in) and idx, score (out; score may be NULL) exactly as for lrsa_score_select.
+ *   - Problems whose scratch need (the score_select figure of lrsa_workspace_bytes) exceeds
+ *     LRSA_STATIC_SCRATCH_BYTES are refused with LRSA_ERR_WORKSPACE_TOO_SMALL and nothing is
+ *     enqueued; use lrsa_score_select with a workspace for those.
+ *   - The device that owns `cuda_stream` must be the current device.  The first call on each device
+ *     looks up the array's device address (once per device); make that first call outside of any
+ *     stream capture.
+ *   - All calls on a device share the one array.  It keeps the previous call's contents; the
+ *     call clears, on the stream, the parts that must start at zero.  Two calls whose kernels could
+ *     overlap on the GPU (different streams without ordering) race on it and give undefined
+ *     results: serialise them.
+ */
+#define LRSA_STATIC_SCRATCH_BYTES (4u << 20)
+int lrsa_score_select_static(const lrsa_params_t* params, const void* K, const void* V, int32_t* idx,
+                             float* score, void* cuda_stream);
+
+/*
  * LRSA attention forward (Section 3.1, Eq. 3 with the chunked mask of Section 3.2).
  * Query position t < S attends positions [0, t].  Query t >= S in chunk c = (t-S)/L attends the
  * sinks, the kept positions idx[b, hkv, w, :] of the first n_c = min(max(c - n_dense_prev, 0),

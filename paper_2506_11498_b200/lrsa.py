@@ -73,6 +73,8 @@ def lib() -> ctypes.CDLL:
         L.lrsa_num_sel_windows.argtypes = [pp, ctypes.POINTER(ctypes.c_int32)]
         L.lrsa_workspace_bytes.argtypes = [pp] + [ctypes.POINTER(sz)] * 3
         L.lrsa_score_select.argtypes = [pp, vp, vp, i32p, fp, vp, sz, vp]
+        L.lrsa_score_select_static.argtypes = [pp, vp, vp, i32p, fp, vp]
+        L.lrsa_score_select_static.restype = ctypes.c_int
         L.lrsa_attn_fwd.argtypes = [pp, vp, vp, vp, i32p, vp, fp, vp, sz, vp]
         L.lrsa_attn_bwd.argtypes = [pp, vp, vp, vp, vp, vp, fp, i32p, vp, vp, vp, vp, sz, vp]
         L.lrsa_workspace_status.argtypes = [vp, vp]
@@ -137,6 +139,20 @@ def lrsa_score_select(params: Params, K, V, idx=None, score=None, workspace=None
     cp = params.c()
     _check(lib().lrsa_score_select(ctypes.byref(cp), _p(K), _p(V), _p(idx), _p(score), _p(workspace),
                                    workspace.numel(), _stream(stream)), "lrsa_score_select")
+    return idx, score
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def lrsa_score_select_static(params: Params, K, V, idx, score=None, stream=None):
+    """lrsa_score_select for callers that cannot provide or allocate scratch memory: the library's
+    own fixed device array (STATIC_SCRATCH_BYTES) is used, so nothing is allocated here either -
+    `idx` (and `score`, if wanted) must be passed in.  Problems that need more scratch raise
+    LRSA_ERR_WORKSPACE_TOO_SMALL.  Calls that may overlap on the GPU must be serialised."""
+    cp = params.c()
+    _check(lib().lrsa_score_select_static(ctypes.byref(cp), _p(K), _p(V), _p(idx), _p(score), _stream(stream)),
+           "lrsa_score_select_static")
     return idx, score
 
 
