@@ -1,0 +1,395 @@
+// LRSA attention forward on tcgen05 tensor cores (Section 3.1 Eq. 3 under the chunked mask of
+// Section 3.2).
+//
+// A CTA owns a block of 256 query rows of one (batch, query head): two 128-row tiles that share one
+// key list (first n_front rows of the compact sinks+kept buffer, then a contiguous range of original
+// positions up to the diagonal).  Roles:
+//   warp 0      TMA producer: Q tiles once, then K_j, V_j tiles through a ring of shared-memory slots
+//   warp 1      MMA issuer:  S_t = Q_t K_j^T (operands in shared memory) and O_t += P_t V_j with P_t
+//               read from tensor memory; owns the TMEM allocation
+//   warps 2-5   softmax of tile 0, warps 6-9 softmax of tile 1: S from TMEM, online softmax in fp32
+//               with the maximum only raised when it grew by more than 2^8 (then O is rescaled in
+//               TMEM), P written back over S as packed bf16
+// While one tile's softmax runs, the tensor core works on the other tile.  All mbarrier waits are
+// bounded; on expiry the CTA records LRSA_ERR_TIMEOUT in the workspace header and leaves.
+#include "attn_common_sm100.h"
+
+namespace lrsa {
+namespace {
+
+using namespace ptx;
+
+template <int D>
+struct FwdCfg {
+  static constexpr int kSub = D / 64;                 // 64-column (128-byte) sub-tiles per tile
+  static constexpr int kSubBytes = kTile * 128;       // 16 KB
+  static constexpr int kTileBytes = kSub * kSubBytes; // one Q / K / V tile
+  static constexpr int kStages = D == 128 ? 5 : 8;    // K/V ring slots
+  static constexpr int kSmem = (2 + kStages) * kTileBytes + 1024;
+  static constexpr int kThreads = 320;
+  static constexpr uint32_t kColS = 0, kColO = 256;   // TMEM columns: S0,S1 then O0,O1
+};
+
+struct FwdArgs {
+  BlockPlan plan;
+  int BH, Hq, Hkv, G, N;
+  __nv_bfloat16* O;
+  float* LSE;
+  float scale, scale_log2;   // softmax scale, and scale * log2(e)
+  int* status;
+};
+
+struct FwdBars {
+  uint64_t q_full;
+  uint64_t kv_full[8], kv_empty[8];
+  uint64_t s_full[2], p_full[2], pv_done[2];
+};
+
+template <int D>
+__global__ void __launch_bounds__(FwdCfg<D>::kThreads, 1)
+lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapKc,
+                const __grid_constant__ CUtensorMap mapVc, const FwdArgs a) {
+  using Cfg = FwdCfg<D>;
+  constexpr int NS = Cfg::kStages;
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) FwdBars bars;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_s;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sQ = smem0, sRing = smem0 + 2 * Cfg::kTileBytes;
+
+  const int bh = blockIdx.x % a.BH, blk = blockIdx.x / a.BH;
+  const RowBlock rb = decode_block(a.plan, blk);
+  const int bh_kv = (bh / a.Hq) * a.Hkv + (bh % a.Hq) / a.G;
+  const int n_ct = (rb.n_front + kTile - 1) / kTile;
+  int n_t[2];
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const int first = rb.q0 + t * kTile;
+    n_t[t] = first >= rb.q_end ? 0 : n_ct + (min(first + kTile - 1, rb.q_end - 1) - rb.dense_start) / kTile + 1;
+  }
+  const int n_max = max(n_t[0], n_t[1]);
+
+  if (tid == 0) {
+    abort_s = 0;
+    mbar_init(smem_u32(&bars.q_full), 1);
+    for (int i = 0; i < NS; ++i) { mbar_init(smem_u32(&bars.kv_full[i]), 1); mbar_init(smem_u32(&bars.kv_empty[i]), 1); }
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(smem_u32(&bars.s_full[t]), 1);
+      mbar_init(smem_u32(&bars.p_full[t]), 128);
+      mbar_init(smem_u32(&bars.pv_done[t]), 1);
+    }
+    fence_barrier_init();
+  }
+  if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_s), 512); tmem_relinquish(); }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_base_s;
+  volatile int* abort = &abort_s;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV);
+      prefetch_tensormap(&mapKc); prefetch_tensormap(&mapVc);
+      mbar_expect_tx(smem_u32(&bars.q_full), 2 * Cfg::kTileBytes);
+      for (int t = 0; t < 2; ++t)
+        for (int h = 0; h < Cfg::kSub; ++h)
+          tma_load_3d(sQ + t * Cfg::kTileBytes + h * Cfg::kSubBytes, &mapQ, h * 64, rb.q0 + t * kTile, bh,
+                      smem_u32(&bars.q_full));
+      int it = 0;
+      bool ok = true;
+      for (int j = 0; j < n_max && ok; ++j) {
+        for (int which = 0; which < 2 && ok; ++which, ++it) {
+          const int slot = it % NS, use = it / NS;
+          if (use > 0) ok = mbar_wait(smem_u32(&bars.kv_empty[slot]), (use - 1) & 1, abort);
+          if (!ok) break;
+          const uint32_t full = smem_u32(&bars.kv_full[slot]);
+          mbar_expect_tx(full, Cfg::kTileBytes);
+          const bool compact = j < n_ct;
+          const CUtensorMap* map = compact ? (which ? &mapVc : &mapKc) : (which ? &mapV : &mapK);
+          const int row = compact ? j * kTile : rb.dense_start + (j - n_ct) * kTile;
+          for (int h = 0; h < Cfg::kSub; ++h)
+            tma_load_3d(sRing + slot * Cfg::kTileBytes + h * Cfg::kSubBytes, map, h * 64, row, bh_kv, full);
+        }
+      }
+      if (!ok) {
+        // give loads already in flight a bounded chance to land before the CTA's smem is released
+        for (int back = 1; back <= NS && back <= it; ++back) {
+          const int i2 = it - back;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(smem_u32(&bars.kv_full[i2 % NS]), (i2 / NS) & 1) && clock64() - t0 < 2000000) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = make_idesc_bf16(kTile, kTile, 0, 0);
+      constexpr uint32_t idesc_pv = make_idesc_bf16(kTile, D, 0, 1);
+      bool ok = mbar_wait(smem_u32(&bars.q_full), 0, abort);
+      for (int j = 0; j <= n_max && ok; ++j) {
+        const int itK = 2 * j, itV = 2 * j - 1;
+        if (j < n_max) ok = mbar_wait(smem_u32(&bars.kv_full[itK % NS]), (itK / NS) & 1, abort);
+        if (ok && j >= 1) ok = mbar_wait(smem_u32(&bars.kv_full[itV % NS]), (itV / NS) & 1, abort);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t sK = sRing + (itK % NS) * Cfg::kTileBytes;
+        const uint32_t sV = sRing + ((itV + NS) % NS) * Cfg::kTileBytes;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          const bool do_qk = j < n_t[t], do_pv = j >= 1 && (j - 1) < n_t[t];
+          if (do_pv) {
+            ok = mbar_wait(smem_u32(&bars.p_full[t]), (j - 1) & 1, abort);
+            if (!ok) break;
+            tc_fence_after_sync();
+#pragma unroll
+            for (int kk = 0; kk < kTile / 16; ++kk)
+              umma_ts(tmem + Cfg::kColO + t * D, tmem + Cfg::kColS + t * kTile + kk * 8,
+                      make_smem_desc_sw128(sV + kk * 2048, Cfg::kSubBytes, 1024), idesc_pv,
+                      (j - 1 > 0 || kk > 0) ? 1u : 0u);
+            umma_commit(smem_u32(&bars.pv_done[t]));
+          }
+          if (do_qk) {
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+              const uint32_t off = (kk >> 2) * Cfg::kSubBytes + (kk & 3) * 32;
+              umma_ss(tmem + Cfg::kColS + t * kTile,
+                      make_smem_desc_sw128(sQ + t * Cfg::kTileBytes + off, 16, 1024),
+                      make_smem_desc_sw128(sK + off, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
+            }
+            umma_commit(smem_u32(&bars.s_full[t]));
+          }
+        }
+        if (!ok) break;
+        if (j < n_max) umma_commit(smem_u32(&bars.kv_empty[itK % NS]));
+        if (j >= 1) umma_commit(smem_u32(&bars.kv_empty[itV % NS]));
+      }
+    }
+  } else {
+    // ---------------- softmax + epilogue ----------------
+    const int t = (warp - 2) >> 2, quad = warp & 3;
+    const int row = quad * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const uint32_t S_addr = tmem + lane_addr + Cfg::kColS + t * kTile;
+    const uint32_t O_addr = tmem + lane_addr + Cfg::kColO + t * D;
+    const int qpos = rb.q0 + t * kTile + row;
+    const int n = n_t[t];
+    const float c = a.scale_log2;
+    float m = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n; ++j) {
+      ok = mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort);
+      if (!ok) break;
+      tc_fence_after_sync();
+      uint32_t s[128];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) tmem_ld32(S_addr + q * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[q * 32]));
+      tmem_wait_ld();
+      const int limit = j < n_ct ? rb.n_front - j * kTile : qpos - (rb.dense_start + (j - n_ct) * kTile) + 1;
+      if (limit < kTile) {
+#pragma unroll
+        for (int i = 0; i < 128; ++i)
+          if (i >= limit) s[i] = 0xff800000u;  // -inf
+      }
+      float mx = __uint_as_float(s[0]);
+#pragma unroll
+      for (int i = 1; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(s[i]));
+      if (j == 0) {
+        m = mx == -INFINITY ? 0.f : mx;
+      } else {
+        const bool need = (mx - m) * c > 8.f;
+        if (__any_sync(0xffffffffu, need)) {
+          ok = mbar_wait(smem_u32(&bars.pv_done[t]), (j - 1) & 1, abort);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const float f = need ? ex2((m - mx) * c) : 1.f;
+#pragma unroll
+          for (int q = 0; q < D / 32; ++q) {
+            uint32_t o[32];
+            tmem_ld32(O_addr + q * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+            tmem_st32(O_addr + q * 32, o);
+          }
+          tmem_wait_st();
+          l *= f;
+          if (need) m = mx;
+        }
+      }
+      const float nmc = -m * c;
+      float sum = 0.f;
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        uint32_t pk[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float p0 = ex2(fmaf(__uint_as_float(s[q * 64 + 2 * i]), c, nmc));
+          const float p1 = ex2(fmaf(__uint_as_float(s[q * 64 + 2 * i + 1]), c, nmc));
+          sum += p0 + p1;
+          pk[i] = pack_bf16(p0, p1);
+        }
+        tmem_st32(S_addr + q * 32, pk);
+      }
+      tmem_wait_st();
+      l += sum;
+      tc_fence_before_sync();
+      mbar_arrive(smem_u32(&bars.p_full[t]));
+    }
+    if (ok && n > 0) {
+      ok = mbar_wait(smem_u32(&bars.pv_done[t]), (n - 1) & 1, abort);
+      if (ok) {
+        tc_fence_after_sync();
+        const float inv = 1.0f / l;
+        const bool store = qpos < rb.q_end;
+        __nv_bfloat16* orow = a.O + ((size_t)bh * a.N + qpos) * D;
+#pragma unroll
+        for (int q = 0; q < D / 32; ++q) {
+          uint32_t o[32];
+          tmem_ld32(O_addr + q * 32, o);
+          tmem_wait_ld();
+          if (store) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              uint4 w;
+              w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+              w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+              w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+              w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+              *reinterpret_cast<uint4*>(orow + q * 32 + v * 8) = w;
+            }
+          }
+        }
+        if (store) a.LSE[(size_t)bh * a.N + qpos] = m * a.scale + logf(l);
+      }
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 512);
+  if (tid == 0 && abort_s) atomicExch(a.status, (int)LRSA_ERR_TIMEOUT);
+}
+
+__global__ void compact_kv_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
+                                  const int32_t* __restrict__ idx, __nv_bfloat16* __restrict__ Kc,
+                                  __nv_bfloat16* __restrict__ Vc, int BHkv, int N, int d, int S, int n_kept, int Rc) {
+  // one warp per compact row; a row is d*2 bytes = 8 (d=128) or 4 (d=64) bytes per lane
+  const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (wid >= (long long)BHkv * Rc) return;
+  const int bh = (int)(wid / Rc), r = (int)(wid % Rc), lane = threadIdx.x & 31;
+  const int pos = r < S ? r : idx[(size_t)bh * n_kept + (r - S)];
+  const size_t src = ((size_t)bh * N + pos) * d, dst = ((size_t)bh * Rc + r) * d;
+  if (d == 128) {
+    reinterpret_cast<uint2*>(Kc + dst)[lane] = reinterpret_cast<const uint2*>(K + src)[lane];
+    reinterpret_cast<uint2*>(Vc + dst)[lane] = reinterpret_cast<const uint2*>(V + src)[lane];
+  } else {
+    reinterpret_cast<uint32_t*>(Kc + dst)[lane] = reinterpret_cast<const uint32_t*>(K + src)[lane];
+    reinterpret_cast<uint32_t*>(Vc + dst)[lane] = reinterpret_cast<const uint32_t*>(V + src)[lane];
+  }
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+  static EncodeFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) p = nullptr;
+    return reinterpret_cast<EncodeFn>(p);
+  }();
+  return fn;
+}
+
+struct FwdWs {
+  size_t kc, vc, total;
+};
+FwdWs fwd_ws_layout(const Geom& g) {
+  FwdWs w;
+  const size_t rc = g.Rc > 0 ? g.Rc : 1;
+  const size_t bytes = align_up((size_t)g.B * g.Hkv * rc * g.d * sizeof(__nv_bfloat16), 1024);
+  w.kc = 1024;
+  w.vc = w.kc + bytes;
+  w.total = w.vc + bytes;
+  return w;
+}
+
+}  // namespace
+
+int make_tmap_bf16(CUtensorMap* map, const void* base, int d, long long rows, long long outer, int box_rows) {
+  EncodeFn fn = encode_fn();
+  if (!fn) return LRSA_ERR_CUDA;
+  cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)outer};
+  cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)d * 2 * (cuuint64_t)rows};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? LRSA_OK : LRSA_ERR_CUDA;
+}
+
+int launch_compact_kv(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat16* V, const int32_t* idx,
+                      __nv_bfloat16* Kc, __nv_bfloat16* Vc, cudaStream_t st) {
+  if (g.Rc == 0) return LRSA_OK;
+  const long long warps = (long long)g.B * g.Hkv * g.Rc;
+  const unsigned blocks = (unsigned)((warps + 7) / 8);
+  compact_kv_kernel<<<blocks, 256, 0, st>>>(K, V, idx, Kc, Vc, g.B * g.Hkv, g.N, g.d, g.S, g.Wsel * g.K, g.Rc);
+  LRSA_CUDA_CHECK(cudaGetLastError());
+  launch_counter().n++;
+  return LRSA_OK;
+}
+
+size_t attn_fwd_ws_bytes(const Geom& g) { return fwd_ws_layout(g).total; }
+
+template <int D>
+static int launch_fwd_t(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K, const __nv_bfloat16* V,
+                        const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, __nv_bfloat16* O, float* LSE, int* status,
+                        cudaStream_t st) {
+  using Cfg = FwdCfg<D>;
+  CUtensorMap mQ, mK, mV, mKc, mVc;
+  const long long rc = g.Rc > 0 ? g.Rc : 1;
+  int rc_ = make_tmap_bf16(&mQ, Q, D, g.N, (long long)g.B * g.Hq, kTile);
+  if (rc_ == LRSA_OK) rc_ = make_tmap_bf16(&mK, K, D, g.N, (long long)g.B * g.Hkv, kTile);
+  if (rc_ == LRSA_OK) rc_ = make_tmap_bf16(&mV, V, D, g.N, (long long)g.B * g.Hkv, kTile);
+  if (rc_ == LRSA_OK) rc_ = make_tmap_bf16(&mKc, Kc, D, rc, (long long)g.B * g.Hkv, kTile);
+  if (rc_ == LRSA_OK) rc_ = make_tmap_bf16(&mVc, Vc, D, rc, (long long)g.B * g.Hkv, kTile);
+  if (rc_ != LRSA_OK) return rc_;
+  FwdArgs a;
+  a.plan = make_plan(g, 2 * kTile);
+  a.BH = g.B * g.Hq; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.N = g.N;
+  a.O = O; a.LSE = LSE; a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f;
+  a.status = status;
+  const long long grid = (long long)a.plan.total * a.BH;
+  if (grid > 0x7fffffffLL) return LRSA_ERR_UNSUPPORTED;
+  auto kern = lrsa_fwd_kernel<D>;
+  LRSA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem));
+  kern<<<(unsigned)grid, Cfg::kThreads, Cfg::kSmem, st>>>(mQ, mK, mV, mKc, mVc, a);
+  LRSA_CUDA_CHECK(cudaGetLastError());
+  launch_counter().n++;
+  return LRSA_OK;
+}
+
+int launch_attn_fwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K, const __nv_bfloat16* V,
+                          const int32_t* idx, __nv_bfloat16* O, float* LSE, void* ws, cudaStream_t st) {
+  const FwdWs lay = fwd_ws_layout(g);
+  unsigned char* base = static_cast<unsigned char*>(ws);
+  LRSA_CUDA_CHECK(cudaMemsetAsync(base, 0, sizeof(WsHeader), st));
+  launch_counter().n++;
+  __nv_bfloat16* Kc = reinterpret_cast<__nv_bfloat16*>(base + lay.kc);
+  __nv_bfloat16* Vc = reinterpret_cast<__nv_bfloat16*>(base + lay.vc);
+  int rc = launch_compact_kv(g, K, V, idx, Kc, Vc, st);
+  if (rc != LRSA_OK) return rc;
+  int* status = &reinterpret_cast<WsHeader*>(base)->status;
+  return g.d == 128 ? launch_fwd_t<128>(g, Q, K, V, Kc, Vc, O, LSE, status, st)
+                    : launch_fwd_t<64>(g, Q, K, V, Kc, Vc, O, LSE, status, st);
+}
+
+}  // namespace lrsa

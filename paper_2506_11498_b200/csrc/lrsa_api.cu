@@ -10,7 +10,7 @@ LaunchCounter& launch_counter() {
   return c;
 }
 
-static int g_impl = 1;  // 0: tensor-core kernels, 1: CUDA-core validation kernels
+static int g_impl = 0;  // 0: tensor-core kernels, 1: CUDA-core validation kernels
 
 int make_geom(const lrsa_params_t* p, Geom* g) {
   if (!p || !g) return LRSA_ERR_INVALID_ARG;
@@ -41,7 +41,10 @@ int make_geom(const lrsa_params_t* p, Geom* g) {
 
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-static size_t fwd_ws_bytes(const Geom& g) { return attn_ref_fwd_ws_bytes(g); }
+static size_t fwd_ws_bytes(const Geom& g) {
+  const size_t a = attn_ref_fwd_ws_bytes(g), b = attn_fwd_ws_bytes(g);
+  return a > b ? a : b;
+}
 static size_t bwd_ws_bytes(const Geom& g) { return attn_ref_bwd_ws_bytes(g); }
 
 }  // namespace lrsa
@@ -99,9 +102,9 @@ int lrsa_attn_fwd(const lrsa_params_t* params, const void* Q, const void* K, con
     return LRSA_ERR_INVALID_ARG;
   if (workspace_bytes < fwd_ws_bytes(g)) return LRSA_ERR_WORKSPACE_TOO_SMALL;
   auto st = static_cast<cudaStream_t>(cuda_stream);
-  return launch_attn_ref_fwd(g, static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
-                             static_cast<const __nv_bfloat16*>(V), idx, static_cast<__nv_bfloat16*>(O), LSE,
-                             workspace, st);
+  auto fn = g_impl == 0 ? launch_attn_fwd_sm100 : launch_attn_ref_fwd;
+  return fn(g, static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
+            static_cast<const __nv_bfloat16*>(V), idx, static_cast<__nv_bfloat16*>(O), LSE, workspace, st);
 }
 
 int lrsa_attn_bwd(const lrsa_params_t* params, const void* Q, const void* K, const void* V,

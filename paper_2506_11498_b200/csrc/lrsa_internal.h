@@ -69,6 +69,12 @@ int launch_attn_ref_bwd(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat
                         const float* LSE, const int32_t* idx, __nv_bfloat16* dQ, __nv_bfloat16* dK,
                         __nv_bfloat16* dV, void* ws, cudaStream_t st);
 
+// attn_fwd_sm100.cu : tcgen05 / TMEM forward (workspace: header + compact K/V).
+size_t attn_fwd_ws_bytes(const Geom& g);
+int launch_attn_fwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
+                          const __nv_bfloat16* V, const int32_t* idx, __nv_bfloat16* O, float* LSE,
+                          void* ws, cudaStream_t st);
+
 #define LRSA_CUDA_CHECK(expr)                                 \
   do {                                                        \
     cudaError_t _e = (expr);                                  \
