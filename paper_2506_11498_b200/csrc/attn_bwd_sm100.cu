@@ -1,0 +1,45 @@
+// LRSA attention backward: workspace layout and the sequence of launches.
+#include "attn_common_sm100.h"
+
+namespace lrsa {
+namespace {
+
+struct BwdWs {
+  size_t kc, vc, dsum, total;
+};
+BwdWs bwd_ws_layout(const Geom& g) {
+  BwdWs w;
+  const size_t rc = g.Rc > 0 ? g.Rc : 1;
+  const size_t cbytes = align_up((size_t)g.B * g.Hkv * rc * g.d * sizeof(__nv_bfloat16), 1024);
+  size_t off = 1024;
+  w.kc = off; off += cbytes;
+  w.vc = off; off += cbytes;
+  w.dsum = off; off += align_up((size_t)g.B * g.Hq * g.N * sizeof(float), 1024);
+  w.total = off;
+  return w;
+}
+
+}  // namespace
+
+size_t attn_bwd_ws_bytes(const Geom& g) { return bwd_ws_layout(g).total; }
+
+int launch_attn_bwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
+                          const __nv_bfloat16* V, const __nv_bfloat16* O, const __nv_bfloat16* dO,
+                          const float* LSE, const int32_t* idx, __nv_bfloat16* dQ, __nv_bfloat16* dK,
+                          __nv_bfloat16* dV, void* ws, cudaStream_t st) {
+  const BwdWs lay = bwd_ws_layout(g);
+  unsigned char* base = static_cast<unsigned char*>(ws);
+  LRSA_CUDA_CHECK(cudaMemsetAsync(base, 0, sizeof(WsHeader), st));
+  launch_counter().n++;
+  __nv_bfloat16* Kc = reinterpret_cast<__nv_bfloat16*>(base + lay.kc);
+  __nv_bfloat16* Vc = reinterpret_cast<__nv_bfloat16*>(base + lay.vc);
+  float* Dsum = reinterpret_cast<float*>(base + lay.dsum);
+  int* status = &reinterpret_cast<WsHeader*>(base)->status;
+  int rc = launch_compact_kv(g, K, V, idx, Kc, Vc, st);
+  if (rc == LRSA_OK) rc = launch_bwd_prep(g, O, dO, Dsum, st);
+  if (rc == LRSA_OK) rc = launch_bwd_dq_sm100(g, Q, dO, K, V, Kc, Vc, LSE, Dsum, dQ, status, st);
+  if (rc == LRSA_OK) rc = launch_attn_ref_bwd_dkv(g, Q, K, V, dO, LSE, idx, Dsum, dK, dV, st);
+  return rc;
+}
+
+}  // namespace lrsa

@@ -232,4 +232,21 @@ int launch_attn_ref_bwd(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat
   return LRSA_OK;
 }
 
+// dK, dV only, with D = rowsum(dO*O) supplied by the caller.
+int launch_attn_ref_bwd_dkv(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
+                            const __nv_bfloat16* V, const __nv_bfloat16* dO, const float* LSE,
+                            const int32_t* idx, const float* Dsum, __nv_bfloat16* dK, __nv_bfloat16* dV,
+                            cudaStream_t st) {
+  RefArgs a = make_args(g);
+  a.Q = Q; a.K = K; a.V = V; a.dO = dO; a.LSE = LSE; a.idx = idx; a.dK = dK; a.dV = dV;
+  a.Dws = const_cast<float*>(Dsum);
+  const long long krows = (long long)g.B * g.Hkv * g.N;
+  const unsigned kb = (unsigned)((krows + 7) / 8);
+  if (g.d == 128) ref_bwd_dkv_kernel<128><<<kb, 256, 0, st>>>(a);
+  else ref_bwd_dkv_kernel<64><<<kb, 256, 0, st>>>(a);
+  LRSA_CUDA_CHECK(cudaGetLastError());
+  launch_counter().n++;
+  return LRSA_OK;
+}
+
 }  // namespace lrsa

@@ -45,7 +45,10 @@ static size_t fwd_ws_bytes(const Geom& g) {
   const size_t a = attn_ref_fwd_ws_bytes(g), b = attn_fwd_ws_bytes(g);
   return a > b ? a : b;
 }
-static size_t bwd_ws_bytes(const Geom& g) { return attn_ref_bwd_ws_bytes(g); }
+static size_t bwd_ws_bytes(const Geom& g) {
+  const size_t a = attn_ref_bwd_ws_bytes(g), b = attn_bwd_ws_bytes(g);
+  return a > b ? a : b;
+}
 
 }  // namespace lrsa
 
@@ -123,9 +126,9 @@ int lrsa_attn_bwd(const lrsa_params_t* params, const void* Q, const void* K, con
   if (workspace_bytes < bwd_ws_bytes(g)) return LRSA_ERR_WORKSPACE_TOO_SMALL;
   auto st = static_cast<cudaStream_t>(cuda_stream);
   auto bf = [](const void* p) { return static_cast<const __nv_bfloat16*>(p); };
-  return launch_attn_ref_bwd(g, bf(Q), bf(K), bf(V), bf(O), bf(dO), LSE, idx,
-                             static_cast<__nv_bfloat16*>(dQ), static_cast<__nv_bfloat16*>(dK),
-                             static_cast<__nv_bfloat16*>(dV), workspace, st);
+  auto fn = g_impl == 0 ? launch_attn_bwd_sm100 : launch_attn_ref_bwd;
+  return fn(g, bf(Q), bf(K), bf(V), bf(O), bf(dO), LSE, idx, static_cast<__nv_bfloat16*>(dQ),
+            static_cast<__nv_bfloat16*>(dK), static_cast<__nv_bfloat16*>(dV), workspace, st);
 }
 
 int lrsa_workspace_status(const void* workspace, void* cuda_stream) {

@@ -75,6 +75,22 @@ int launch_attn_fwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bflo
                           const __nv_bfloat16* V, const int32_t* idx, __nv_bfloat16* O, float* LSE,
                           void* ws, cudaStream_t st);
 
+int launch_attn_ref_bwd_dkv(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
+                            const __nv_bfloat16* V, const __nv_bfloat16* dO, const float* LSE,
+                            const int32_t* idx, const float* Dsum, __nv_bfloat16* dK, __nv_bfloat16* dV,
+                            cudaStream_t st);
+
+// attn_bwd_*_sm100.cu : tcgen05 / TMEM backward.
+size_t attn_bwd_ws_bytes(const Geom& g);
+int launch_attn_bwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
+                          const __nv_bfloat16* V, const __nv_bfloat16* O, const __nv_bfloat16* dO,
+                          const float* LSE, const int32_t* idx, __nv_bfloat16* dQ, __nv_bfloat16* dK,
+                          __nv_bfloat16* dV, void* ws, cudaStream_t st);
+int launch_bwd_prep(const Geom& g, const __nv_bfloat16* O, const __nv_bfloat16* dO, float* Dsum, cudaStream_t st);
+int launch_bwd_dq_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO, const __nv_bfloat16* K,
+                        const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, const float* LSE,
+                        const float* Dsum, __nv_bfloat16* dQ, int* status, cudaStream_t st);
+
 #define LRSA_CUDA_CHECK(expr)                                 \
   do {                                                        \
     cudaError_t _e = (expr);                                  \
