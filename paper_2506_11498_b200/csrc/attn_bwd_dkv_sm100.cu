@@ -1,0 +1,489 @@
+// LRSA attention backward, dK / dV part, on tcgen05 tensor cores (key-outer).
+//
+// The keys of one (batch, KV head) are cut into 128-row tiles of two kinds:
+//   compact tiles : rows of the compact sinks+kept buffer; seen by every query of the chunks that
+//                   see those windows compressed
+//   dense tiles   : original positions of one window (or of the sink region / the tail); seen
+//                   causally by the queries from the diagonal to the end of the last chunk that
+//                   still sees that window uncompressed
+// A CTA takes one tile and a segment of its (query head of the group, 64-row query tile) list:
+//   S^T  = K_j Q_i^T     (smem x smem -> TMEM, keys on lanes)     P^T  = exp2(S^T*c - LSE_i*log2e)
+//   dP^T = V_j dO_i^T    (smem x smem -> TMEM)                    dS^T = P^T * (dP^T - D_i)
+//   dV  += P^T dO_i      (TMEM x smem -> TMEM)
+//   dK  += dS^T Q_i      (TMEM x smem -> TMEM)
+// P^T and dS^T are written back over S^T and dP^T as packed bf16; both are double-buffered so the
+// tensor core computes the next S^T/dP^T while one warpgroup handles the current pair.  At the end
+// the accumulators are added (fp32 atomics) to a zeroed workspace indexed by original position
+// (dense tiles) or by compact row (compact tiles); two small kernels then fold the compact rows
+// onto their original positions and convert to bf16.
+#include "attn_common_sm100.h"
+
+namespace lrsa {
+namespace {
+
+using namespace ptx;
+
+constexpr int kQRows = 64;    // query rows per inner tile
+constexpr int kSeg = 256;     // inner iterations per CTA at most
+
+struct DkvPlan {
+  int S, L, K, N, W, T, C, Wsel, ndp, Rc, G;
+  int n_cmp;       // compact tiles
+  int n_sink;      // dense tiles of the sink region
+  int per_win;     // dense tiles per full window
+  int per_tail;    // dense tiles of the tail
+  int n_tiles;
+};
+
+struct KvTile {
+  int kind;      // 0 compact, 1 dense
+  int row0;      // first compact row / first key position
+  int key_end;   // rows at or beyond this are not part of the tile
+  int qb, qend;  // query positions [qb, qend) see (part of) the tile
+  int nq;        // 64-row query tiles per head
+};
+
+inline DkvPlan make_dkv_plan(const Geom& g) {
+  DkvPlan p;
+  p.S = g.S; p.L = g.L; p.K = g.K; p.N = g.N; p.W = g.W; p.T = g.T; p.C = g.C; p.Wsel = g.Wsel;
+  p.ndp = g.ndp; p.Rc = g.Rc; p.G = g.G;
+  p.n_cmp = (g.Rc + kTile - 1) / kTile;
+  p.n_sink = (g.S + kTile - 1) / kTile;
+  p.per_win = (g.L + kTile - 1) / kTile;
+  p.per_tail = (g.T + kTile - 1) / kTile;
+  p.n_tiles = p.n_cmp + p.n_sink + g.W * p.per_win + p.per_tail;
+  return p;
+}
+
+__host__ __device__ inline KvTile describe_tile(const DkvPlan& p, int tile) {
+  KvTile t;
+  if (tile < p.n_cmp) {
+    t.kind = 0;
+    t.row0 = tile * kTile;
+    t.key_end = p.Rc;
+    int cmin = 0;
+    if (t.row0 >= p.S) cmin = first_compressed_chunk((t.row0 - p.S) / p.K, p.ndp, p.Wsel, p.C);
+    t.qb = p.S + cmin * p.L;
+    t.qend = cmin >= p.C ? t.qb : p.N;
+  } else {
+    t.kind = 1;
+    int d = tile - p.n_cmp;
+    if (d < p.n_sink) {
+      t.row0 = d * kTile; t.key_end = p.S; t.qend = p.S;
+    } else {
+      d -= p.n_sink;
+      int w;
+      if (d < p.W * p.per_win) {
+        w = d / p.per_win;
+        t.row0 = p.S + w * p.L + (d % p.per_win) * kTile;
+        t.key_end = p.S + (w + 1) * p.L;
+      } else {
+        w = p.W;
+        t.row0 = p.S + p.W * p.L + (d - p.W * p.per_win) * kTile;
+        t.key_end = p.N;
+      }
+      const int cc = first_compressed_chunk(w, p.ndp, p.Wsel, p.C);
+      t.qend = cc >= p.C ? p.N : (p.S + cc * p.L < p.N ? p.S + cc * p.L : p.N);
+    }
+    t.qb = t.row0;
+  }
+  t.nq = t.qend > t.qb ? (t.qend - t.qb + kQRows - 1) / kQRows : 0;
+  return t;
+}
+
+__host__ __device__ inline int tile_segments(const DkvPlan& p, const KvTile& t) {
+  return (p.G * t.nq + kSeg - 1) / kSeg;
+}
+
+// seg_prefix[i] = number of segments of tiles < i   (one block)
+__global__ void dkv_setup_kernel(const DkvPlan p, int* seg_prefix) {
+  for (int i = threadIdx.x; i < p.n_tiles; i += blockDim.x)
+    seg_prefix[i + 1] = tile_segments(p, describe_tile(p, i));
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int acc = 0;
+    seg_prefix[0] = 0;
+    for (int i = 1; i <= p.n_tiles; ++i) { acc += seg_prefix[i]; seg_prefix[i] = acc; }
+  }
+}
+
+template <int D>
+struct DkvCfg {
+  static constexpr int kSub = D / 64;
+  static constexpr int kKSubBytes = kTile * 128;            // 128 key rows x 128 bytes
+  static constexpr int kKTileBytes = kSub * kKSubBytes;     // K_j or V_j
+  static constexpr int kQSubBytes = kQRows * 128;           // 64 query rows x 128 bytes
+  static constexpr int kQTileBytes = kSub * kQSubBytes;     // Q_i or dO_i
+  static constexpr int kStageBytes = 2 * kQTileBytes;       // Q_i + dO_i
+  static constexpr int kStages = D == 128 ? 4 : 8;
+  static constexpr int kSmem = 2 * kKTileBytes + kStages * kStageBytes + 1024;
+  static constexpr int kThreads = 320;
+  static constexpr uint32_t kColS = 0, kColP = 128, kColK = 256, kColV = 256 + D;
+};
+
+struct DkvArgs {
+  DkvPlan plan;
+  int BHkv, Hq, Hkv, total_segs;
+  const float* LSE;
+  const float* Dsum;
+  const int* seg_prefix;
+  float* dKf;   // [BHkv][N + Rc][D] fp32, zeroed
+  float* dVf;
+  int rows_ws;  // N + Rc
+  float scale, scale_log2;
+  int* status;
+};
+
+struct DkvBars {
+  uint64_t kv_full, acc_done;
+  uint64_t ring_full[8], ring_empty[8];
+  uint64_t s_full[2], p_full[2];
+};
+
+__device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+template <int D>
+__global__ void __launch_bounds__(DkvCfg<D>::kThreads, 1)
+lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapdO,
+                    const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
+                    const __grid_constant__ CUtensorMap mapKc, const __grid_constant__ CUtensorMap mapVc,
+                    const DkvArgs a) {
+  using Cfg = DkvCfg<D>;
+  constexpr int NS = Cfg::kStages;
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) DkvBars bars;
+  __shared__ __align__(16) float st_nl2[NS][kQRows];   // -LSE*log2(e) per query row of the stage (-inf: not seen)
+  __shared__ __align__(16) float st_D[NS][kQRows];
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_s;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sK = smem0, sV = smem0 + Cfg::kKTileBytes, sRing = smem0 + 2 * Cfg::kKTileBytes;
+
+  // ---- which tile, which segment ----
+  const DkvPlan& p = a.plan;
+  const int bh_kv = blockIdx.x % a.BHkv, seg = blockIdx.x / a.BHkv;
+  int lo_t = 0, hi_t = p.n_tiles;   // last tile with seg_prefix[tile] <= seg
+  while (hi_t - lo_t > 1) {
+    const int mid = (lo_t + hi_t) >> 1;
+    if (a.seg_prefix[mid] <= seg) lo_t = mid; else hi_t = mid;
+  }
+  const KvTile kt = describe_tile(p, lo_t);
+  const int it_begin = (seg - a.seg_prefix[lo_t]) * kSeg;
+  const int n = min(kSeg, p.G * kt.nq - it_begin);
+  const int hq0 = (bh_kv / a.Hkv) * a.Hq + (bh_kv % a.Hkv) * p.G;   // first query head of the group
+
+  if (tid == 0) {
+    abort_s = 0;
+    mbar_init(smem_u32(&bars.kv_full), 1);
+    mbar_init(smem_u32(&bars.acc_done), 1);
+    for (int i = 0; i < NS; ++i) { mbar_init(smem_u32(&bars.ring_full[i]), 1); mbar_init(smem_u32(&bars.ring_empty[i]), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&bars.s_full[b]), 1); mbar_init(smem_u32(&bars.p_full[b]), 128); }
+    fence_barrier_init();
+  }
+  if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_s), 512); tmem_relinquish(); }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_base_s;
+  volatile int* abort = &abort_s;
+
+  if (warp == 0) {
+    // ---------------- producer (whole warp: lanes stage LSE and D, lane 0 drives TMA) ----------------
+    if (lane == 0) {
+      prefetch_tensormap(&mapQ); prefetch_tensormap(&mapdO);
+      const CUtensorMap* mk = kt.kind == 0 ? &mapKc : &mapK;
+      const CUtensorMap* mv = kt.kind == 0 ? &mapVc : &mapV;
+      mbar_expect_tx(smem_u32(&bars.kv_full), 2 * Cfg::kKTileBytes);
+      for (int h = 0; h < Cfg::kSub; ++h) {
+        tma_load_3d(sK + h * Cfg::kKSubBytes, mk, h * 64, kt.row0, bh_kv, smem_u32(&bars.kv_full));
+        tma_load_3d(sV + h * Cfg::kKSubBytes, mv, h * 64, kt.row0, bh_kv, smem_u32(&bars.kv_full));
+      }
+    }
+    bool ok = true;
+    int it = 0;
+    for (; it < n; ++it) {
+      const int slot = it % NS, use = it / NS;
+      if (use > 0 && lane == 0) ok = mbar_wait(smem_u32(&bars.ring_empty[slot]), (use - 1) & 1, abort);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      const int gi = it_begin + it;
+      const int hq = hq0 + gi / kt.nq, q0 = kt.qb + (gi % kt.nq) * kQRows;
+      for (int r = lane; r < kQRows; r += 32) {
+        const int q = q0 + r;
+        const bool seen = q < kt.qend;
+        st_nl2[slot][r] = seen ? -a.LSE[(size_t)hq * p.N + q] * 1.4426950408889634f : -INFINITY;
+        st_D[slot][r] = seen ? a.Dsum[(size_t)hq * p.N + q] : 0.f;
+      }
+      __syncwarp();
+      if (lane == 0) {
+        const uint32_t full = smem_u32(&bars.ring_full[slot]);
+        mbar_expect_tx(full, Cfg::kStageBytes);
+        const uint32_t dst = sRing + slot * Cfg::kStageBytes;
+        for (int h = 0; h < Cfg::kSub; ++h) {
+          tma_load_3d(dst + h * Cfg::kQSubBytes, &mapQ, h * 64, q0, hq, full);
+          tma_load_3d(dst + Cfg::kQTileBytes + h * Cfg::kQSubBytes, &mapdO, h * 64, q0, hq, full);
+        }
+      }
+    }
+    if (!ok && lane == 0) {
+      for (int back = 1; back <= NS && back <= it; ++back) {
+        const int i2 = it - back;
+        const long long t0 = clock64();
+        while (!mbar_try_wait(smem_u32(&bars.ring_full[i2 % NS]), (i2 / NS) & 1) && clock64() - t0 < 2000000) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kQRows, 0, 0);  // S^T, dP^T : 128 keys x 64 queries
+      constexpr uint32_t idesc_a = make_idesc_bf16(kTile, D, 0, 1);       // dV, dK    : 128 keys x D
+      bool ok = mbar_wait(smem_u32(&bars.kv_full), 0, abort);
+      for (int it = 0; it <= n && ok; ++it) {
+        if (it < n) {
+          const int slot = it % NS, b = it & 1;
+          ok = mbar_wait(smem_u32(&bars.ring_full[slot]), (it / NS) & 1, abort);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t sQi = sRing + slot * Cfg::kStageBytes, sdOi = sQi + Cfg::kQTileBytes;
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t koff = (kk >> 2) * Cfg::kKSubBytes + (kk & 3) * 32;
+            const uint32_t qoff = (kk >> 2) * Cfg::kQSubBytes + (kk & 3) * 32;
+            umma_ss(tmem + Cfg::kColS + b * kQRows, make_smem_desc_sw128(sK + koff, 16, 1024),
+                    make_smem_desc_sw128(sQi + qoff, 16, 1024), idesc_s, kk > 0 ? 1u : 0u);
+          }
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t koff = (kk >> 2) * Cfg::kKSubBytes + (kk & 3) * 32;
+            const uint32_t qoff = (kk >> 2) * Cfg::kQSubBytes + (kk & 3) * 32;
+            umma_ss(tmem + Cfg::kColP + b * kQRows, make_smem_desc_sw128(sV + koff, 16, 1024),
+                    make_smem_desc_sw128(sdOi + qoff, 16, 1024), idesc_s, kk > 0 ? 1u : 0u);
+          }
+          umma_commit(smem_u32(&bars.s_full[b]));
+        }
+        if (it >= 1) {
+          const int pi = it - 1, slot = pi % NS, b = pi & 1;
+          ok = mbar_wait(smem_u32(&bars.p_full[b]), (pi >> 1) & 1, abort);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t sQi = sRing + slot * Cfg::kStageBytes, sdOi = sQi + Cfg::kQTileBytes;
+#pragma unroll
+          for (int kk = 0; kk < kQRows / 16; ++kk)
+            umma_ts(tmem + Cfg::kColV, tmem + Cfg::kColS + b * kQRows + kk * 8,
+                    make_smem_desc_sw128(sdOi + kk * 2048, Cfg::kQSubBytes, 1024), idesc_a, (pi > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+          for (int kk = 0; kk < kQRows / 16; ++kk)
+            umma_ts(tmem + Cfg::kColK, tmem + Cfg::kColP + b * kQRows + kk * 8,
+                    make_smem_desc_sw128(sQi + kk * 2048, Cfg::kQSubBytes, 1024), idesc_a, (pi > 0 || kk > 0) ? 1u : 0u);
+          umma_commit(smem_u32(&bars.ring_empty[slot]));
+        }
+      }
+      if (ok) umma_commit(smem_u32(&bars.acc_done));
+    }
+  } else {
+    // ---------------- P^T / dS^T warpgroups + epilogue ----------------
+    const int wg = (warp - 2) >> 2, quad = warp & 3;
+    const int r = quad * 32 + lane;            // key row of this thread inside the tile
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const float c = a.scale_log2;
+    const bool key_ok = kt.row0 + r < kt.key_end;
+    bool ok = true;
+    for (int it = wg; it < n; it += 2) {
+      const int slot = it % NS;
+      ok = mbar_wait(smem_u32(&bars.s_full[wg]), (it >> 1) & 1, abort);
+      if (ok) ok = mbar_wait(smem_u32(&bars.ring_full[slot]), (it / NS) & 1, abort);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t S_addr = tmem + lane_addr + Cfg::kColS + wg * kQRows;
+      const uint32_t P_addr = tmem + lane_addr + Cfg::kColP + wg * kQRows;
+      uint32_t s[64], dp[64];
+      tmem_ld32(S_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+      tmem_ld32(S_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+      tmem_ld32(P_addr, *reinterpret_cast<uint32_t(*)[32]>(&dp[0]));
+      tmem_ld32(P_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&dp[32]));
+      tmem_wait_ld();
+      // first query column of this tile that sees this thread's key (64 = none)
+      const int gi = it_begin + it;
+      const int q0 = kt.qb + (gi % kt.nq) * kQRows;
+      int lo;
+      if (!key_ok) {
+        lo = kQRows;
+      } else if (kt.kind == 1) {
+        lo = kt.row0 + r - q0;                      // causal: query position >= key position
+      } else {
+        const int cr = kt.row0 + r;                 // compact row: needs cr < S + n_hist(chunk)*K
+        lo = kQRows;
+        int col = 0;
+        while (col < kQRows) {
+          const int cch = (q0 + col - p.S) / p.L;
+          if (cr < p.S + n_hist_windows(cch, p.ndp, p.Wsel) * p.K) { lo = col; break; }
+          col = p.S + (cch + 1) * p.L - q0;         // first column of the next chunk
+        }
+      }
+      if (lo > 0) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i)
+          if (i < lo) s[i] = 0xff800000u;
+      }
+      const float4* nl2v = reinterpret_cast<const float4*>(st_nl2[slot]);
+      const float4* Dv = reinterpret_cast<const float4*>(st_D[slot]);
+      uint32_t pp[32], ds[32];
+#pragma unroll
+      for (int v = 0; v < 16; ++v) {
+        const float4 nl = nl2v[v], dd = Dv[v];
+        const float p0 = ex2(fmaf(__uint_as_float(s[4 * v + 0]), c, nl.x));
+        const float p1 = ex2(fmaf(__uint_as_float(s[4 * v + 1]), c, nl.y));
+        const float p2 = ex2(fmaf(__uint_as_float(s[4 * v + 2]), c, nl.z));
+        const float p3 = ex2(fmaf(__uint_as_float(s[4 * v + 3]), c, nl.w));
+        pp[2 * v] = pack_bf16(p0, p1);
+        pp[2 * v + 1] = pack_bf16(p2, p3);
+        ds[2 * v] = pack_bf16(p0 * (__uint_as_float(dp[4 * v + 0]) - dd.x), p1 * (__uint_as_float(dp[4 * v + 1]) - dd.y));
+        ds[2 * v + 1] = pack_bf16(p2 * (__uint_as_float(dp[4 * v + 2]) - dd.z), p3 * (__uint_as_float(dp[4 * v + 3]) - dd.w));
+      }
+      tmem_st32(S_addr, pp);
+      tmem_st32(P_addr, ds);
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(smem_u32(&bars.p_full[wg]));
+    }
+    if (ok) ok = mbar_wait(smem_u32(&bars.acc_done), 0, abort);
+    if (ok) {
+      tc_fence_after_sync();
+      // warpgroup 0 adds dK (scaled), warpgroup 1 adds dV
+      const uint32_t acc = tmem + lane_addr + (wg == 0 ? Cfg::kColK : Cfg::kColV);
+      const float mul = wg == 0 ? a.scale : 1.0f;
+      const int out_row = kt.kind == 0 ? p.N + kt.row0 + r : kt.row0 + r;
+      float* dst = (wg == 0 ? a.dKf : a.dVf) + ((size_t)bh_kv * a.rows_ws + out_row) * D;
+#pragma unroll
+      for (int q = 0; q < D / 32; ++q) {
+        uint32_t o[32];
+        tmem_ld32(acc + q * 32, o);
+        tmem_wait_ld();
+        if (key_ok) {
+#pragma unroll
+          for (int v = 0; v < 8; ++v)
+            red_add_v4(dst + q * 32 + v * 4, __uint_as_float(o[4 * v]) * mul, __uint_as_float(o[4 * v + 1]) * mul,
+                       __uint_as_float(o[4 * v + 2]) * mul, __uint_as_float(o[4 * v + 3]) * mul);
+        }
+      }
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 512);
+  if (tid == 0 && abort_s) atomicExch(a.status, (int)LRSA_ERR_TIMEOUT);
+}
+
+// dense[pos(r)] += compact[r] for every compact row (positions are distinct), one warp per row
+__global__ void fold_compact_kernel(float* dKf, float* dVf, const int32_t* __restrict__ idx, int BHkv, int N, int Rc,
+                                    int S, int n_kept, int d) {
+  const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (wid >= (long long)BHkv * Rc) return;
+  const int bh = (int)(wid / Rc), r = (int)(wid % Rc), lane = threadIdx.x & 31;
+  const int pos = r < S ? r : idx[(size_t)bh * n_kept + (r - S)];
+  const size_t base = (size_t)bh * (N + Rc);
+  for (int c = lane; c < d; c += 32) {
+    dKf[(base + pos) * d + c] += dKf[(base + N + r) * d + c];
+    dVf[(base + pos) * d + c] += dVf[(base + N + r) * d + c];
+  }
+}
+
+// bf16 outputs from the fp32 accumulation rows [0, N) of every (batch, KV head)
+__global__ void convert_dkv_kernel(const float* __restrict__ dKf, const float* __restrict__ dVf,
+                                   __nv_bfloat16* __restrict__ dK, __nv_bfloat16* __restrict__ dV, long long n4,
+                                   long long row_elems_out, long long row_elems_ws) {
+  // n4 = number of float4 groups over [BHkv][N][d]; row_elems_* = N*d and (N+Rc)*d
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n4) return;
+  const long long e = i * 4, bh = e / row_elems_out, off = e % row_elems_out;
+  const float4 k = *reinterpret_cast<const float4*>(dKf + bh * row_elems_ws + off);
+  const float4 v = *reinterpret_cast<const float4*>(dVf + bh * row_elems_ws + off);
+  uint2 ko, vo;
+  ko.x = pack_bf16(k.x, k.y); ko.y = pack_bf16(k.z, k.w);
+  vo.x = pack_bf16(v.x, v.y); vo.y = pack_bf16(v.z, v.w);
+  *reinterpret_cast<uint2*>(dK + e) = ko;
+  *reinterpret_cast<uint2*>(dV + e) = vo;
+}
+
+}  // namespace
+
+size_t dkv_ws_bytes(const Geom& g, size_t* prefix_bytes) {
+  const DkvPlan p = make_dkv_plan(g);
+  const size_t pre = align_up((size_t)(p.n_tiles + 1) * sizeof(int), 1024);
+  if (prefix_bytes) *prefix_bytes = pre;
+  const size_t acc = align_up((size_t)g.B * g.Hkv * (g.N + g.Rc) * g.d * sizeof(float), 1024);
+  return pre + 2 * acc;
+}
+
+template <int D>
+static int launch_dkv_t(const Geom& g, const DkvArgs& a, const CUtensorMap* m, cudaStream_t st) {
+  using Cfg = DkvCfg<D>;
+  auto kern = lrsa_bwd_dkv_kernel<D>;
+  LRSA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem));
+  const long long grid = (long long)a.total_segs * a.BHkv;
+  if (grid > 0x7fffffffLL) return LRSA_ERR_UNSUPPORTED;
+  if (grid == 0) return LRSA_OK;
+  kern<<<(unsigned)grid, Cfg::kThreads, Cfg::kSmem, st>>>(m[0], m[1], m[2], m[3], m[4], m[5], a);
+  LRSA_CUDA_CHECK(cudaGetLastError());
+  launch_counter().n++;
+  return LRSA_OK;
+}
+
+// ws_dkv: region of dkv_ws_bytes(g) bytes.  Zeroes the accumulators, runs the tile kernel, folds the
+// compact rows onto their positions and writes bf16 dK, dV.
+int launch_bwd_dkv_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO, const __nv_bfloat16* K,
+                         const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, const float* LSE,
+                         const float* Dsum, const int32_t* idx, __nv_bfloat16* dK, __nv_bfloat16* dV, void* ws_dkv,
+                         int* status, cudaStream_t st) {
+  const DkvPlan p = make_dkv_plan(g);
+  size_t pre = 0;
+  const size_t total = dkv_ws_bytes(g, &pre);
+  unsigned char* base = static_cast<unsigned char*>(ws_dkv);
+  const size_t acc = (total - pre) / 2;
+  int* seg_prefix = reinterpret_cast<int*>(base);
+  float* dKf = reinterpret_cast<float*>(base + pre);
+  float* dVf = reinterpret_cast<float*>(base + pre + acc);
+  LRSA_CUDA_CHECK(cudaMemsetAsync(base + pre, 0, 2 * acc, st));
+  launch_counter().n++;
+  dkv_setup_kernel<<<1, 256, 0, st>>>(p, seg_prefix);
+  LRSA_CUDA_CHECK(cudaGetLastError());
+  launch_counter().n++;
+  int total_segs = 0;
+  for (int i = 0; i < p.n_tiles; ++i) total_segs += tile_segments(p, describe_tile(p, i));
+
+  CUtensorMap m[6];
+  const long long rc = g.Rc > 0 ? g.Rc : 1;
+  int r = make_tmap_bf16(&m[0], Q, g.d, g.N, (long long)g.B * g.Hq, kQRows);
+  if (r == LRSA_OK) r = make_tmap_bf16(&m[1], dO, g.d, g.N, (long long)g.B * g.Hq, kQRows);
+  if (r == LRSA_OK) r = make_tmap_bf16(&m[2], K, g.d, g.N, (long long)g.B * g.Hkv, kTile);
+  if (r == LRSA_OK) r = make_tmap_bf16(&m[3], V, g.d, g.N, (long long)g.B * g.Hkv, kTile);
+  if (r == LRSA_OK) r = make_tmap_bf16(&m[4], Kc, g.d, rc, (long long)g.B * g.Hkv, kTile);
+  if (r == LRSA_OK) r = make_tmap_bf16(&m[5], Vc, g.d, rc, (long long)g.B * g.Hkv, kTile);
+  if (r != LRSA_OK) return r;
+  DkvArgs a;
+  a.plan = p; a.BHkv = g.B * g.Hkv; a.Hq = g.Hq; a.Hkv = g.Hkv; a.total_segs = total_segs;
+  a.LSE = LSE; a.Dsum = Dsum; a.seg_prefix = seg_prefix; a.dKf = dKf; a.dVf = dVf; a.rows_ws = g.N + g.Rc;
+  a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f; a.status = status;
+  r = g.d == 128 ? launch_dkv_t<128>(g, a, m, st) : launch_dkv_t<64>(g, a, m, st);
+  if (r != LRSA_OK) return r;
+  if (g.Rc > 0) {
+    const long long warps = (long long)a.BHkv * g.Rc;
+    fold_compact_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(dKf, dVf, idx, a.BHkv, g.N, g.Rc, g.S,
+                                                                    g.Wsel * g.K, g.d);
+    LRSA_CUDA_CHECK(cudaGetLastError());
+    launch_counter().n++;
+  }
+  const long long n4 = (long long)a.BHkv * g.N * g.d / 4;
+  convert_dkv_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(dKf, dVf, dK, dV, n4, (long long)g.N * g.d,
+                                                                  (long long)(g.N + g.Rc) * g.d);
+  LRSA_CUDA_CHECK(cudaGetLastError());
+  launch_counter().n++;
+  return LRSA_OK;
+}
+
+}  // namespace lrsa

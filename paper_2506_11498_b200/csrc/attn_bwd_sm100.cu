@@ -5,7 +5,7 @@ namespace lrsa {
 namespace {
 
 struct BwdWs {
-  size_t kc, vc, dsum, total;
+  size_t kc, vc, dsum, dkv, total;
 };
 BwdWs bwd_ws_layout(const Geom& g) {
   BwdWs w;
@@ -15,6 +15,7 @@ BwdWs bwd_ws_layout(const Geom& g) {
   w.kc = off; off += cbytes;
   w.vc = off; off += cbytes;
   w.dsum = off; off += align_up((size_t)g.B * g.Hq * g.N * sizeof(float), 1024);
+  w.dkv = off; off += dkv_ws_bytes(g, nullptr);
   w.total = off;
   return w;
 }
@@ -38,7 +39,8 @@ int launch_attn_bwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bflo
   int rc = launch_compact_kv(g, K, V, idx, Kc, Vc, st);
   if (rc == LRSA_OK) rc = launch_bwd_prep(g, O, dO, Dsum, st);
   if (rc == LRSA_OK) rc = launch_bwd_dq_sm100(g, Q, dO, K, V, Kc, Vc, LSE, Dsum, dQ, status, st);
-  if (rc == LRSA_OK) rc = launch_attn_ref_bwd_dkv(g, Q, K, V, dO, LSE, idx, Dsum, dK, dV, st);
+  if (rc == LRSA_OK)
+    rc = launch_bwd_dkv_sm100(g, Q, dO, K, V, Kc, Vc, LSE, Dsum, idx, dK, dV, base + lay.dkv, status, st);
   return rc;
 }
 
