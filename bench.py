@@ -156,12 +156,11 @@ def oracle_sample(w, n_chunks=3, host=None):
 
 def run_reference(args, w):
     """Reference arm: the CPU checker on host cores, each step a bounded sample."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    from paper_2506_11498_b200 import replicas, workloads
+    if replicas.env_rank_world()[0] != 0:
         return
     f_fwd, f_bwd = flops(w)
     vals = []
-    from paper_2506_11498_b200 import workloads
     host = workloads.generate(w)
     for i in range(args.warmup + args.steps):
         s = oracle_sample(w, n_chunks=2, host=host)
@@ -188,8 +187,8 @@ def run_reference(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_32k_gqa7_d128")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -204,11 +203,9 @@ def main():
         return
 
     import torch
-    from paper_2506_11498_b200 import lrsa
+    from paper_2506_11498_b200 import lrsa, replicas
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = replicas.env_rank_world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
     torch.cuda.set_device(local)
@@ -217,7 +214,7 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     # weak scaling: every rank runs its own sequence (independent problems, no data-path collective)
-    wl = w.with_(seed=w.seed + 1000 * rank)
+    wl = replicas.rank_workload(w, rank)
     lrsa.lib()
     p = lrsa.Params.from_workload(wl)
     host = {k: v.pin_memory() for k, v in workloads.generate(wl).items()}
@@ -278,11 +275,7 @@ def main():
     t_fwd = [e[1].elapsed_time(e[2]) for e in timers]
     t_bwd = [e[2].elapsed_time(e[3]) for e in timers]
     t_step = [e[0].elapsed_time(e[3]) for e in timers]
-    total_ms = sum(t_step)
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = replicas.max_over_ranks(sum(t_step), dist, "cuda")
     ms_per_step = total_ms / args.steps
 
     # end to end through the C ABI with HOST buffers: H2D of Q,K,V,dO from pinned memory and D2H
@@ -310,13 +303,9 @@ def main():
             e2e_step()
         e1.record(stream)
         barrier()
-        e2e_ms = e0.elapsed_time(e1) / n_e2e
-        if dist is not None:
-            t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = replicas.max_over_ranks(e0.elapsed_time(e1) / n_e2e, dist, "cuda")
         f_fwd, f_bwd = flops(wl)
-        e2e = {"value": world * (f_fwd + f_bwd) / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+        e2e = {"value": replicas.job_rate(f_fwd + f_bwd, world, e2e_ms * 1e-3) / 1e12, "unit": UNIT,
                "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     if rank != 0:
@@ -332,7 +321,7 @@ def main():
     peak_tf = peaks["bf16_tflops_sustained"]
     achieved = f_bwd / bwd_s / 1e12
     line = {
-        "metric": METRIC, "value": world * (f_fwd + f_bwd) / (ms_per_step * 1e-3) / 1e12, "unit": UNIT,
+        "metric": METRIC, "value": replicas.job_rate(f_fwd + f_bwd, world, ms_per_step * 1e-3) / 1e12, "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
