@@ -124,8 +124,7 @@ struct DkvCfg {
 struct DkvArgs {
   DkvPlan plan;
   int BHkv, Hq, Hkv, total_segs;
-  const float* LSE;
-  const float* Dsum;
+  const float2* stats;   // per query row: (-LSE * log2(e), D)
   const int* seg_prefix;
   float* dKf;   // [BHkv][N + Rc][D] fp32, zeroed
   float* dVf;
@@ -205,18 +204,32 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     }
     bool ok = true;
     int it = 0;
+    // per-row statistics of a stage are fetched one stage ahead, so that their latency overlaps the
+    // wait for a free slot instead of adding to it
+    auto fetch = [&](int i, float2 (&v)[kQRows / 32]) {
+      const int gi = it_begin + i;
+      const int hq = hq0 + gi / kt.nq, q0 = kt.qb + (gi % kt.nq) * kQRows;
+#pragma unroll
+      for (int k = 0; k < kQRows / 32; ++k) {
+        const int q = q0 + lane + 32 * k;
+        v[k] = q < kt.qend ? __ldg(a.stats + (size_t)hq * p.N + q) : make_float2(-INFINITY, 0.f);
+      }
+    };
+    float2 cur[kQRows / 32], nxt[kQRows / 32];
+    if (n > 0) fetch(0, cur);
     for (; it < n; ++it) {
       const int slot = it % NS, use = it / NS;
+      if (it + 1 < n) fetch(it + 1, nxt);
       if (use > 0 && lane == 0) ok = mbar_wait(smem_u32(&bars.ring_empty[slot]), (use - 1) & 1, abort);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       const int gi = it_begin + it;
       const int hq = hq0 + gi / kt.nq, q0 = kt.qb + (gi % kt.nq) * kQRows;
-      for (int r = lane; r < kQRows; r += 32) {
-        const int q = q0 + r;
-        const bool seen = q < kt.qend;
-        st_nl2[slot][r] = seen ? -a.LSE[(size_t)hq * p.N + q] * 1.4426950408889634f : -INFINITY;
-        st_D[slot][r] = seen ? a.Dsum[(size_t)hq * p.N + q] : 0.f;
+#pragma unroll
+      for (int k = 0; k < kQRows / 32; ++k) {
+        st_nl2[slot][lane + 32 * k] = cur[k].x;
+        st_D[slot][lane + 32 * k] = cur[k].y;
+        cur[k] = nxt[k];
       }
       __syncwarp();
       if (lane == 0) {
@@ -237,53 +250,64 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kQRows, 0, 0);  // S^T, dP^T : 128 keys x 64 queries
-      constexpr uint32_t idesc_a = make_idesc_bf16(kTile, D, 0, 1);       // dV, dK    : 128 keys x D
-      bool ok = mbar_wait(smem_u32(&bars.kv_full), 0, abort);
-      for (int it = 0; it <= n && ok; ++it) {
-        if (it < n) {
-          const int slot = it % NS, b = it & 1;
-          ok = mbar_wait(smem_u32(&bars.ring_full[slot]), (it / NS) & 1, abort);
-          if (!ok) break;
-          tc_fence_after_sync();
-          const uint32_t sQi = sRing + slot * Cfg::kStageBytes, sdOi = sQi + Cfg::kQTileBytes;
+    // ---------------- MMA issuer: the whole warp runs the loop, one elected lane issues ----------------
+    constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kQRows, 0, 0);  // S^T, dP^T : 128 keys x 64 queries
+    constexpr uint32_t idesc_a = make_idesc_bf16(kTile, D, 0, 1);       // dV, dK    : 128 keys x D
+    const uint64_t descK = make_smem_desc_sw128(sK, 16, 1024), descV = make_smem_desc_sw128(sV, 16, 1024);
+    const uint64_t descR = make_smem_desc_sw128(sRing, 16, 1024);                    // K-major Q_i / dO_i
+    const uint64_t descRmn = make_smem_desc_sw128(sRing, Cfg::kQSubBytes, 1024);     // MN-major Q_i / dO_i
+    bool ok = mbar_wait_warp(smem_u32(&bars.kv_full), 0, abort);
+    for (int it = 0; it <= n && ok; ++it) {
+      if (it < n) {
+        const int slot = it % NS, b = it & 1;
+        ok = mbar_wait_warp(smem_u32(&bars.ring_full[slot]), (it / NS) & 1, abort);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint64_t dQi = desc_advance(descR, slot * Cfg::kStageBytes);
+        const uint64_t ddOi = desc_advance(dQi, Cfg::kQTileBytes);
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t koff = (kk >> 2) * Cfg::kKSubBytes + (kk & 3) * 32;
-            const uint32_t qoff = (kk >> 2) * Cfg::kQSubBytes + (kk & 3) * 32;
-            umma_ss(tmem + Cfg::kColS + b * kQRows, make_smem_desc_sw128(sK + koff, 16, 1024),
-                    make_smem_desc_sw128(sQi + qoff, 16, 1024), idesc_s, kk > 0 ? 1u : 0u);
-          }
-#pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t koff = (kk >> 2) * Cfg::kKSubBytes + (kk & 3) * 32;
-            const uint32_t qoff = (kk >> 2) * Cfg::kQSubBytes + (kk & 3) * 32;
-            umma_ss(tmem + Cfg::kColP + b * kQRows, make_smem_desc_sw128(sV + koff, 16, 1024),
-                    make_smem_desc_sw128(sdOi + qoff, 16, 1024), idesc_s, kk > 0 ? 1u : 0u);
-          }
-          umma_commit(smem_u32(&bars.s_full[b]));
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t koff = (kk >> 2) * Cfg::kKSubBytes + (kk & 3) * 32;
+          const uint32_t qoff = (kk >> 2) * Cfg::kQSubBytes + (kk & 3) * 32;
+          const uint64_t ad = desc_advance(descK, koff), bd = desc_advance(dQi, qoff);
+          if (elect_one()) umma_ss(tmem + Cfg::kColS + b * kQRows, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
         }
-        if (it >= 1) {
-          const int pi = it - 1, slot = pi % NS, b = pi & 1;
-          ok = mbar_wait(smem_u32(&bars.p_full[b]), (pi >> 1) & 1, abort);
-          if (!ok) break;
-          tc_fence_after_sync();
-          const uint32_t sQi = sRing + slot * Cfg::kStageBytes, sdOi = sQi + Cfg::kQTileBytes;
 #pragma unroll
-          for (int kk = 0; kk < kQRows / 16; ++kk)
-            umma_ts(tmem + Cfg::kColV, tmem + Cfg::kColS + b * kQRows + kk * 8,
-                    make_smem_desc_sw128(sdOi + kk * 2048, Cfg::kQSubBytes, 1024), idesc_a, (pi > 0 || kk > 0) ? 1u : 0u);
-#pragma unroll
-          for (int kk = 0; kk < kQRows / 16; ++kk)
-            umma_ts(tmem + Cfg::kColK, tmem + Cfg::kColP + b * kQRows + kk * 8,
-                    make_smem_desc_sw128(sQi + kk * 2048, Cfg::kQSubBytes, 1024), idesc_a, (pi > 0 || kk > 0) ? 1u : 0u);
-          umma_commit(smem_u32(&bars.ring_empty[slot]));
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t koff = (kk >> 2) * Cfg::kKSubBytes + (kk & 3) * 32;
+          const uint32_t qoff = (kk >> 2) * Cfg::kQSubBytes + (kk & 3) * 32;
+          const uint64_t ad = desc_advance(descV, koff), bd = desc_advance(ddOi, qoff);
+          if (elect_one()) umma_ss(tmem + Cfg::kColP + b * kQRows, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
         }
+        if (elect_one()) umma_commit(smem_u32(&bars.s_full[b]));
+        __syncwarp();
       }
-      if (ok) umma_commit(smem_u32(&bars.acc_done));
+      if (it >= 1) {
+        const int pi = it - 1, slot = pi % NS, b = pi & 1;
+        ok = mbar_wait_warp(smem_u32(&bars.p_full[b]), (pi >> 1) & 1, abort);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint64_t dQi = desc_advance(descRmn, slot * Cfg::kStageBytes);
+        const uint64_t ddOi = desc_advance(dQi, Cfg::kQTileBytes);
+        const uint32_t acc0 = pi > 0 ? 1u : 0u;
+#pragma unroll
+        for (int kk = 0; kk < kQRows / 16; ++kk) {
+          const uint64_t bd = desc_advance(ddOi, kk * 2048);
+          if (elect_one())
+            umma_ts(tmem + Cfg::kColV, tmem + Cfg::kColS + b * kQRows + kk * 8, bd, idesc_a, kk > 0 ? 1u : acc0);
+        }
+#pragma unroll
+        for (int kk = 0; kk < kQRows / 16; ++kk) {
+          const uint64_t bd = desc_advance(dQi, kk * 2048);
+          if (elect_one())
+            umma_ts(tmem + Cfg::kColK, tmem + Cfg::kColP + b * kQRows + kk * 8, bd, idesc_a, kk > 0 ? 1u : acc0);
+        }
+        if (elect_one()) umma_commit(smem_u32(&bars.ring_empty[slot]));
+        __syncwarp();
+      }
     }
+    if (ok && elect_one()) umma_commit(smem_u32(&bars.acc_done));
+    __syncwarp();
   } else {
     // ---------------- P^T / dS^T warpgroups + epilogue ----------------
     const int wg = (warp - 2) >> 2, quad = warp & 3;
@@ -437,8 +461,8 @@ static int launch_dkv_t(const Geom& g, const DkvArgs& a, const CUtensorMap* m, c
 // ws_dkv: region of dkv_ws_bytes(g) bytes.  Zeroes the accumulators, runs the tile kernel, folds the
 // compact rows onto their positions and writes bf16 dK, dV.
 int launch_bwd_dkv_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO, const __nv_bfloat16* K,
-                         const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, const float* LSE,
-                         const float* Dsum, const int32_t* idx, __nv_bfloat16* dK, __nv_bfloat16* dV, void* ws_dkv,
+                         const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, const float2* stats,
+                         const int32_t* idx, __nv_bfloat16* dK, __nv_bfloat16* dV, void* ws_dkv,
                          int* status, cudaStream_t st) {
   const DkvPlan p = make_dkv_plan(g);
   size_t pre = 0;
@@ -467,7 +491,7 @@ int launch_bwd_dkv_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloa
   if (r != LRSA_OK) return r;
   DkvArgs a;
   a.plan = p; a.BHkv = g.B * g.Hkv; a.Hq = g.Hq; a.Hkv = g.Hkv; a.total_segs = total_segs;
-  a.LSE = LSE; a.Dsum = Dsum; a.seg_prefix = seg_prefix; a.dKf = dKf; a.dVf = dVf; a.rows_ws = g.N + g.Rc;
+  a.stats = stats; a.seg_prefix = seg_prefix; a.dKf = dKf; a.dVf = dVf; a.rows_ws = g.N + g.Rc;
   a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f; a.status = status;
   r = g.d == 128 ? launch_dkv_t<128>(g, a, m, st) : launch_dkv_t<64>(g, a, m, st);
   if (r != LRSA_OK) return r;

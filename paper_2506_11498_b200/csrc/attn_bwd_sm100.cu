@@ -5,7 +5,7 @@ namespace lrsa {
 namespace {
 
 struct BwdWs {
-  size_t kc, vc, dsum, dkv, total;
+  size_t kc, vc, stats, dkv, total;
 };
 BwdWs bwd_ws_layout(const Geom& g) {
   BwdWs w;
@@ -14,7 +14,7 @@ BwdWs bwd_ws_layout(const Geom& g) {
   size_t off = 1024;
   w.kc = off; off += cbytes;
   w.vc = off; off += cbytes;
-  w.dsum = off; off += align_up((size_t)g.B * g.Hq * g.N * sizeof(float), 1024);
+  w.stats = off; off += align_up((size_t)g.B * g.Hq * g.N * sizeof(float2), 1024);
   w.dkv = off; off += dkv_ws_bytes(g, nullptr);
   w.total = off;
   return w;
@@ -34,13 +34,13 @@ int launch_attn_bwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bflo
   launch_counter().n++;
   __nv_bfloat16* Kc = reinterpret_cast<__nv_bfloat16*>(base + lay.kc);
   __nv_bfloat16* Vc = reinterpret_cast<__nv_bfloat16*>(base + lay.vc);
-  float* Dsum = reinterpret_cast<float*>(base + lay.dsum);
+  float2* stats = reinterpret_cast<float2*>(base + lay.stats);
   int* status = &reinterpret_cast<WsHeader*>(base)->status;
   int rc = launch_compact_kv(g, K, V, idx, Kc, Vc, st);
-  if (rc == LRSA_OK) rc = launch_bwd_prep(g, O, dO, Dsum, st);
-  if (rc == LRSA_OK) rc = launch_bwd_dq_sm100(g, Q, dO, K, V, Kc, Vc, LSE, Dsum, dQ, status, st);
+  if (rc == LRSA_OK) rc = launch_bwd_prep(g, O, dO, LSE, stats, st);
+  if (rc == LRSA_OK) rc = launch_bwd_dq_sm100(g, Q, dO, K, V, Kc, Vc, stats, dQ, status, st);
   if (rc == LRSA_OK)
-    rc = launch_bwd_dkv_sm100(g, Q, dO, K, V, Kc, Vc, LSE, Dsum, idx, dK, dV, base + lay.dkv, status, st);
+    rc = launch_bwd_dkv_sm100(g, Q, dO, K, V, Kc, Vc, stats, idx, dK, dV, base + lay.dkv, status, st);
   return rc;
 }
 

@@ -24,6 +24,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// The same wait executed by all 32 lanes of a converged warp, with one verdict for the warp.  The
+// warps that issue tcgen05.mma run in warp-uniform control flow with descriptors computed once
+// outside the loops (building a descriptor per instruction in a single-lane branch costs ~100
+// cycles per MMA, more than the MMA itself) and elect one lane per instruction.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort) {
+  const bool ok = mbar_wait(bar, parity, abort);
+  return __all_sync(0xffffffffu, ok);
+}
+
 // A block of query rows that share one key list: rows [q0, q_end) (at most `rows_per_block`), all in
 // one query chunk (or the sink region).  Their keys are the first n_front rows of the compact
 // (sinks + kept) buffer followed by original positions [dense_start, own position].

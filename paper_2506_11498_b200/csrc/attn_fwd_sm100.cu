@@ -127,48 +127,56 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      constexpr uint32_t idesc_qk = make_idesc_bf16(kTile, kTile, 0, 0);
-      constexpr uint32_t idesc_pv = make_idesc_bf16(kTile, D, 0, 1);
-      bool ok = mbar_wait(smem_u32(&bars.q_full), 0, abort);
-      for (int j = 0; j <= n_max && ok; ++j) {
-        const int itK = 2 * j, itV = 2 * j - 1;
-        if (j < n_max) ok = mbar_wait(smem_u32(&bars.kv_full[itK % NS]), (itK / NS) & 1, abort);
-        if (ok && j >= 1) ok = mbar_wait(smem_u32(&bars.kv_full[itV % NS]), (itV / NS) & 1, abort);
-        if (!ok) break;
-        tc_fence_after_sync();
-        const uint32_t sK = sRing + (itK % NS) * Cfg::kTileBytes;
-        const uint32_t sV = sRing + ((itV + NS) % NS) * Cfg::kTileBytes;
+    // ---------------- MMA issuer: the whole warp runs the loop, one elected lane issues ----------------
+    constexpr uint32_t idesc_qk = make_idesc_bf16(kTile, kTile, 0, 0);
+    constexpr uint32_t idesc_pv = make_idesc_bf16(kTile, D, 0, 1);
+    const uint64_t descQ = make_smem_desc_sw128(sQ, 16, 1024);
+    const uint64_t descK0 = make_smem_desc_sw128(sRing, 16, 1024);
+    const uint64_t descV0 = make_smem_desc_sw128(sRing, Cfg::kSubBytes, 1024);
+    bool ok = mbar_wait_warp(smem_u32(&bars.q_full), 0, abort);
+    for (int j = 0; j <= n_max && ok; ++j) {
+      const int itK = 2 * j, itV = 2 * j - 1;
+      if (j < n_max) ok = mbar_wait_warp(smem_u32(&bars.kv_full[itK % NS]), (itK / NS) & 1, abort);
+      if (ok && j >= 1) ok = mbar_wait_warp(smem_u32(&bars.kv_full[itV % NS]), (itV / NS) & 1, abort);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint64_t dK = desc_advance(descK0, (itK % NS) * Cfg::kTileBytes);
+      const uint64_t dV = desc_advance(descV0, ((itV + NS) % NS) * Cfg::kTileBytes);
 #pragma unroll
-        for (int t = 0; t < 2; ++t) {
-          const bool do_qk = j < n_t[t], do_pv = j >= 1 && (j - 1) < n_t[t];
-          if (do_pv) {
-            ok = mbar_wait(smem_u32(&bars.p_full[t]), (j - 1) & 1, abort);
-            if (!ok) break;
+      for (int t = 0; t < 2; ++t) {
+        const bool do_qk = j < n_t[t], do_pv = j >= 1 && (j - 1) < n_t[t];
+        if (do_pv && ok) {
+          ok = mbar_wait_warp(smem_u32(&bars.p_full[t]), (j - 1) & 1, abort);
+          if (ok) {
             tc_fence_after_sync();
+            const uint32_t acc0 = j - 1 > 0 ? 1u : 0u;
 #pragma unroll
-            for (int kk = 0; kk < kTile / 16; ++kk)
-              umma_ts(tmem + Cfg::kColO + t * D, tmem + Cfg::kColS + t * kTile + kk * 8,
-                      make_smem_desc_sw128(sV + kk * 2048, Cfg::kSubBytes, 1024), idesc_pv,
-                      (j - 1 > 0 || kk > 0) ? 1u : 0u);
-            umma_commit(smem_u32(&bars.pv_done[t]));
-          }
-          if (do_qk) {
-#pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-              const uint32_t off = (kk >> 2) * Cfg::kSubBytes + (kk & 3) * 32;
-              umma_ss(tmem + Cfg::kColS + t * kTile,
-                      make_smem_desc_sw128(sQ + t * Cfg::kTileBytes + off, 16, 1024),
-                      make_smem_desc_sw128(sK + off, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
+            for (int kk = 0; kk < kTile / 16; ++kk) {
+              const uint64_t bd = desc_advance(dV, kk * 2048);
+              if (elect_one())
+                umma_ts(tmem + Cfg::kColO + t * D, tmem + Cfg::kColS + t * kTile + kk * 8, bd, idesc_pv,
+                        kk > 0 ? 1u : acc0);
             }
-            umma_commit(smem_u32(&bars.s_full[t]));
+            if (elect_one()) umma_commit(smem_u32(&bars.pv_done[t]));
+            __syncwarp();
           }
         }
-        if (!ok) break;
-        if (j < n_max) umma_commit(smem_u32(&bars.kv_empty[itK % NS]));
-        if (j >= 1) umma_commit(smem_u32(&bars.kv_empty[itV % NS]));
+        if (do_qk && ok) {
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = (kk >> 2) * Cfg::kSubBytes + (kk & 3) * 32;
+            const uint64_t ad = desc_advance(descQ, t * Cfg::kTileBytes + off), bd = desc_advance(dK, off);
+            if (elect_one()) umma_ss(tmem + Cfg::kColS + t * kTile, ad, bd, idesc_qk, kk > 0 ? 1u : 0u);
+          }
+          if (elect_one()) umma_commit(smem_u32(&bars.s_full[t]));
+          __syncwarp();
+        }
       }
+      if (!ok) break;
+      if (j < n_max && elect_one()) umma_commit(smem_u32(&bars.kv_empty[itK % NS]));
+      __syncwarp();
+      if (j >= 1 && elect_one()) umma_commit(smem_u32(&bars.kv_empty[itV % NS]));
+      __syncwarp();
     }
   } else {
     // ---------------- softmax + epilogue ----------------

@@ -74,6 +74,8 @@ ATTN_CASES = [
     (W("a_ndp0_two", 1, 2, 2, 4 + 2 * 256 + 10, 64, 256, 16, 4, seed=29), 0),
     (W("a_one_token", 1, 1, 1, 1, 64, 8, 2, 0, seed=30), 1),
     (W("a_sinks_only", 1, 2, 1, 5, 64, 8, 2, 5, seed=31), 1),
+    (W("a_offsets", 1, 4, 2, 4 + 5 * 256 + 77, 128, 256, 64, 4, seed=32, values="channel_offset"), 1),
+    (W("a_salient64", 1, 4, 1, 16 + 5 * 128 + 40, 64, 128, 32, 16, seed=33, values="salient"), 1),
 ]
 
 
