@@ -124,7 +124,8 @@ struct DkvCfg {
 struct DkvArgs {
   DkvPlan plan;
   int BHkv, Hq, Hkv, total_segs;
-  const float2* stats;   // per query row: (-LSE * log2(e), D)
+  const float2* stats;   // per query row: (-LSE * log2(e), D~ = rowsum(dO * O) from the bf16 O)
+  float* Dacc;           // [B*Hq][N], zeroed: receives sum_j P_tj dP_tj, the accurate D for the dQ kernel
   const int* seg_prefix;
   float* dKf;   // [BHkv][N + Rc][D] fp32, zeroed
   float* dVf;
@@ -356,6 +357,7 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
       const float4* nl2v = reinterpret_cast<const float4*>(st_nl2[slot]);
       const float4* Dv = reinterpret_cast<const float4*>(st_D[slot]);
       uint32_t pp[32], ds[32];
+      float x[64];   // P * dP, whose sum over the keys is the accurate D of the query column
 #pragma unroll
       for (int v = 0; v < 16; ++v) {
         const float4 nl = nl2v[v], dd = Dv[v];
@@ -363,16 +365,37 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         const float p1 = ex2(fmaf(__uint_as_float(s[4 * v + 1]), c, nl.y));
         const float p2 = ex2(fmaf(__uint_as_float(s[4 * v + 2]), c, nl.z));
         const float p3 = ex2(fmaf(__uint_as_float(s[4 * v + 3]), c, nl.w));
+        const float g0 = __uint_as_float(dp[4 * v + 0]), g1 = __uint_as_float(dp[4 * v + 1]);
+        const float g2 = __uint_as_float(dp[4 * v + 2]), g3 = __uint_as_float(dp[4 * v + 3]);
         pp[2 * v] = pack_bf16(p0, p1);
         pp[2 * v + 1] = pack_bf16(p2, p3);
-        ds[2 * v] = pack_bf16(p0 * (__uint_as_float(dp[4 * v + 0]) - dd.x), p1 * (__uint_as_float(dp[4 * v + 1]) - dd.y));
-        ds[2 * v + 1] = pack_bf16(p2 * (__uint_as_float(dp[4 * v + 2]) - dd.z), p3 * (__uint_as_float(dp[4 * v + 3]) - dd.w));
+        ds[2 * v] = pack_bf16(p0 * (g0 - dd.x), p1 * (g1 - dd.y));
+        ds[2 * v + 1] = pack_bf16(p2 * (g2 - dd.z), p3 * (g3 - dd.w));
+        x[4 * v + 0] = p0 * g0; x[4 * v + 1] = p1 * g1; x[4 * v + 2] = p2 * g2; x[4 * v + 3] = p3 * g3;
       }
       tmem_st32(S_addr, pp);
       tmem_st32(P_addr, ds);
       tmem_wait_st();
       tc_fence_before_sync();
       mbar_arrive(smem_u32(&bars.p_full[wg]));
+      // Off the tensor core's critical path: sum x over the warp's 32 keys by halving exchanges; lane l
+      // ends with query columns 2l and 2l+1, which it adds to the per-row accumulator in global memory.
+#pragma unroll
+      for (int m = 32, bit = 16; m >= 2; m >>= 1, bit >>= 1) {
+        const bool up = (lane & bit) != 0;
+#pragma unroll
+        for (int i = 0; i < m; ++i) {
+          const float send = up ? x[i] : x[i + m];
+          const float keep = up ? x[i + m] : x[i];
+          x[i] = keep + __shfl_xor_sync(0xffffffffu, send, bit);
+        }
+      }
+      {
+        const int hq = hq0 + gi / kt.nq;
+        float* drow = a.Dacc + (size_t)hq * p.N + q0 + 2 * lane;
+        if (q0 + 2 * lane < kt.qend) atomicAdd(drow, x[0]);
+        if (q0 + 2 * lane + 1 < kt.qend) atomicAdd(drow + 1, x[1]);
+      }
     }
     if (ok) ok = mbar_wait(smem_u32(&bars.acc_done), 0, abort);
     if (ok) {
@@ -462,7 +485,7 @@ static int launch_dkv_t(const Geom& g, const DkvArgs& a, const CUtensorMap* m, c
 // compact rows onto their positions and writes bf16 dK, dV.
 int launch_bwd_dkv_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO, const __nv_bfloat16* K,
                          const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, const float2* stats,
-                         const int32_t* idx, __nv_bfloat16* dK, __nv_bfloat16* dV, void* ws_dkv,
+                         float* Dacc, const int32_t* idx, __nv_bfloat16* dK, __nv_bfloat16* dV, void* ws_dkv,
                          int* status, cudaStream_t st) {
   const DkvPlan p = make_dkv_plan(g);
   size_t pre = 0;
@@ -491,7 +514,7 @@ int launch_bwd_dkv_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloa
   if (r != LRSA_OK) return r;
   DkvArgs a;
   a.plan = p; a.BHkv = g.B * g.Hkv; a.Hq = g.Hq; a.Hkv = g.Hkv; a.total_segs = total_segs;
-  a.stats = stats; a.seg_prefix = seg_prefix; a.dKf = dKf; a.dVf = dVf; a.rows_ws = g.N + g.Rc;
+  a.stats = stats; a.Dacc = Dacc; a.seg_prefix = seg_prefix; a.dKf = dKf; a.dVf = dVf; a.rows_ws = g.N + g.Rc;
   a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f; a.status = status;
   r = g.d == 128 ? launch_dkv_t<128>(g, a, m, st) : launch_dkv_t<64>(g, a, m, st);
   if (r != LRSA_OK) return r;

@@ -1,20 +1,24 @@
 // LRSA attention backward, dQ part, on tcgen05 tensor cores.
 //
 // A CTA owns one 128-row query tile of one (batch, query head) and walks its key list (the same
-// row-block decomposition as the forward) in 64-key tiles.  Per key tile j:
-//   S  = Q K_j^T          (smem x smem -> TMEM)      P  = exp2(S*c - LSE*log2e)
-//   dP = dO V_j^T         (smem x smem -> TMEM)      dS = P * (dP - D~)         (bf16, back into TMEM)
-//   A += dS K_j           (TMEM x smem -> TMEM)      M += P K_j                 (TMEM x smem -> TMEM)
-// S/dP are double-buffered in TMEM: the two softmax warpgroups alternate over key tiles, so the
-// tensor core computes S/dP of tile j+1 while tile j is in the softmax.
+// row-block decomposition as the forward) in 64-key tiles.  Q and dO are copied once into tensor
+// memory, so every product takes its 128-row operand from TMEM and only the K_j / V_j tiles from
+// shared memory (with both operands in shared memory the kernel is bound by shared-memory
+// bandwidth, not by the tensor core).  Per key tile j:
+//   S  = Q K_j^T          (TMEM x smem -> TMEM)      P  = exp2(S*c - LSE*log2e)
+//   dP = dO V_j^T         (TMEM x smem -> TMEM)      dS = P * (dP - D)          (bf16, back into TMEM)
+//   A += dS K_j           (TMEM x smem -> TMEM)      epilogue: dQ = scale * (A - r * kbar) -> bf16
+// S/dP are double-buffered in TMEM, so the tensor core computes tile j+1 while tile j is in the
+// softmax; both softmax warpgroups work on every tile (32 key columns each) to keep the latency
+// between "S ready" and "dS ready" short.  Warps: 0 TMA producer, 1-3 tensor-core issuers (S, dP, A;
+// no warp has more than eight tcgen05.mma per tile to issue), 4-11 softmax and epilogue.
 //
-// D~ = rowsum(dO * O) comes from the bf16 O and is therefore only approximate; its error, and the
-// bf16 rounding of dS, would be multiplied by the softmax-averaged key M_t = sum_j P_tj k_j, which is
-// large when keys have outlier channels or a few salient keys dominate the row.  Rows of the exact dS
-// sum to zero, so the epilogue removes whatever the rounded rows sum to:
-//   dQ_t = scale * (A_t - r_t * M_t),  r_t = sum_j bf16(dS_tj)       (= scale * sum_j dS_tj (k_j - M_t))
-// which cancels the error of D~ exactly and centres the rounding errors.  The kernel also writes the
-// accurate D_t = sum_j P_tj dP_tj (fp32, thread-local) for the dK/dV kernel that runs after it.
+// D_t = sum_j P_tj dP_tj comes from the dK/dV kernel, which runs first and accumulates it in fp32
+// (rowsum(dO * O) of the bf16 O is not accurate enough: its error is multiplied by the
+// softmax-averaged key, which is large when a few salient keys dominate a row).
+// Rows of the exact dS sum to zero; after bf16 rounding they sum to r_t, which multiplies whatever
+// constant vector the keys of a head share (outlier channels).  The epilogue subtracts r_t * kbar,
+// kbar the mean key of the KV head; in exact arithmetic this subtracts zero.
 #include "attn_common_sm100.h"
 
 namespace lrsa {
@@ -33,24 +37,27 @@ struct DqCfg {
   static constexpr int kKTileBytes = kSub * kKSubBytes;    // one K or V tile
   static constexpr int kStages = D == 128 ? 9 : 16;        // ring slots, K and V tiles alternate
   static constexpr int kSmem = 2 * kQTileBytes + kStages * kKTileBytes + 1024;
-  static constexpr int kThreads = 320;
-  // TMEM columns: buffer b holds S at b*128 and dP at b*128+64; accumulators A at 256, M at 256+D
-  static constexpr uint32_t kColP = 64, kColA = 256, kColM = 256 + D;
+  static constexpr int kThreads = 384;
+  // TMEM columns: Q and dO as packed bf16 (D/2 columns each), accumulator A at D, then buffer b with
+  // S at 256 + 128b and dP 64 columns further
+  static constexpr uint32_t kColQ = 0, kColdO = D / 2, kColA = D, kColBuf = 256, kColP = 64;
 };
 
 struct DqArgs {
   BlockPlan plan;
   int BH, Hq, Hkv, G, N;
-  float2* stats;   // per query row: in (-LSE*log2e, D~); out: .y replaced by the accurate D
+  const float2* stats;   // per query row: (-LSE*log2e, D~); only the first component is used here
+  const float* Dacc;     // per query row: D = sum_j P dP
+  const float* kbar;     // [B*Hkv][D] mean key
   __nv_bfloat16* dQ;
   float scale, scale_log2;
   int* status;
 };
 
 struct DqBars {
-  uint64_t q_full, acc_done;
+  uint64_t q_full, qt_ready, acc_done;
   uint64_t kv_full[16], kv_empty[16];
-  uint64_t s_full[2], p_full[2];
+  uint64_t s_full[2], p_full[2], buf_free[2];
 };
 
 template <int D>
@@ -63,7 +70,7 @@ lrsa_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
   constexpr int NS = Cfg::kStages;
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) DqBars bars;
-  __shared__ float red_s[2][2][kTile];   // [warpgroup][D partial, r partial][row]
+  __shared__ float red_s[2][kTile];   // [column half][row] sums of the rounded dS
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
 
@@ -80,9 +87,14 @@ lrsa_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
   if (tid == 0) {
     abort_s = 0;
     mbar_init(smem_u32(&bars.q_full), 1);
+    mbar_init(smem_u32(&bars.qt_ready), 256);
     mbar_init(smem_u32(&bars.acc_done), 1);
     for (int i = 0; i < NS; ++i) { mbar_init(smem_u32(&bars.kv_full[i]), 1); mbar_init(smem_u32(&bars.kv_empty[i]), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&bars.s_full[b]), 1); mbar_init(smem_u32(&bars.p_full[b]), 128); }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars.s_full[b]), 2);      // the S issuer and the dP issuer
+      mbar_init(smem_u32(&bars.p_full[b]), 256);    // every softmax thread
+      mbar_init(smem_u32(&bars.buf_free[b]), 1);
+    }
     fence_barrier_init();
   }
   if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_s), 512); tmem_relinquish(); }
@@ -127,138 +139,139 @@ lrsa_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
         }
       }
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer: the whole warp runs the loop, one elected lane issues ----------------
-    constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kKeys, 0, 0);   // S, dP : 128 x 64
-    constexpr uint32_t idesc_a = make_idesc_bf16(kTile, D, 0, 1);       // A, M  : 128 x D, B = K_j MN-major
-    const uint64_t descQ = make_smem_desc_sw128(sQ, 16, 1024), descdO = make_smem_desc_sw128(sdO, 16, 1024);
-    const uint64_t descR = make_smem_desc_sw128(sRing, 16, 1024);                  // K-major K_j / V_j
-    const uint64_t descRmn = make_smem_desc_sw128(sRing, Cfg::kKSubBytes, 1024);   // MN-major K_j
-    bool ok = mbar_wait_warp(smem_u32(&bars.q_full), 0, abort);
-    // ring order: K_j at 2j, V_j at 2j+1.  Iteration j issues S/dP of tile j, then A/M of tile j-1.
-    for (int j = 0; j <= n && ok; ++j) {
-      if (j < n) {
-        const int itK = 2 * j, itV = 2 * j + 1, b = j & 1;
-        ok = mbar_wait_warp(smem_u32(&bars.kv_full[itK % NS]), (itK / NS) & 1, abort);
-        if (ok) ok = mbar_wait_warp(smem_u32(&bars.kv_full[itV % NS]), (itV / NS) & 1, abort);
-        if (!ok) break;
-        tc_fence_after_sync();
-        const uint64_t dK = desc_advance(descR, (itK % NS) * Cfg::kKTileBytes);
-        const uint64_t dV = desc_advance(descR, (itV % NS) * Cfg::kKTileBytes);
+  } else if (warp == 1 || warp == 2) {
+    // ---------------- S issuer (warp 1: Q K_j^T) and dP issuer (warp 2: dO V_j^T) ----------------
+    // Each issuing warp runs its loop with all lanes (uniform control flow, descriptors computed once)
+    // and elects one lane per instruction.
+    const int which = warp - 1;                                          // 0: K tiles, 1: V tiles
+    constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kKeys, 0, 0);   // 128 x 64
+    const uint64_t descR = make_smem_desc_sw128(sRing, 16, 1024);       // K-major K_j / V_j
+    const uint32_t a_tmem = tmem + (which == 0 ? Cfg::kColQ : Cfg::kColdO);
+    bool ok = mbar_wait_warp(smem_u32(&bars.qt_ready), 0, abort);   // Q and dO are in tensor memory
+    for (int j = 0; j < n && ok; ++j) {
+      const int it = 2 * j + which, b = j & 1;   // ring order: K_j at 2j, V_j at 2j+1
+      ok = mbar_wait_warp(smem_u32(&bars.kv_full[it % NS]), (it / NS) & 1, abort);
+      if (ok && j >= 2) ok = mbar_wait_warp(smem_u32(&bars.buf_free[b]), ((j >> 1) - 1) & 1, abort);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t d_tmem = tmem + Cfg::kColBuf + b * 128 + which * Cfg::kColP;
+      const uint64_t dT = desc_advance(descR, (it % NS) * Cfg::kKTileBytes);
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t qoff = (kk >> 2) * Cfg::kQSubBytes + (kk & 3) * 32;
-          const uint32_t koff = (kk >> 2) * Cfg::kKSubBytes + (kk & 3) * 32;
-          const uint64_t ad = desc_advance(descQ, qoff), bd = desc_advance(dK, koff);
-          if (elect_one()) umma_ss(tmem + b * kTile, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
-        }
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t qoff = (kk >> 2) * Cfg::kQSubBytes + (kk & 3) * 32;
-          const uint32_t koff = (kk >> 2) * Cfg::kKSubBytes + (kk & 3) * 32;
-          const uint64_t ad = desc_advance(descdO, qoff), bd = desc_advance(dV, koff);
-          if (elect_one()) umma_ss(tmem + b * kTile + Cfg::kColP, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
-        }
-        if (elect_one()) {
-          umma_commit(smem_u32(&bars.s_full[b]));
-          umma_commit(smem_u32(&bars.kv_empty[itV % NS]));   // V_j is used by dP only
-        }
-        __syncwarp();
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const uint64_t bd = desc_advance(dT, (kk >> 2) * Cfg::kKSubBytes + (kk & 3) * 32);
+        if (elect_one()) umma_ts(d_tmem, a_tmem + kk * 8, bd, idesc_s, kk > 0 ? 1u : 0u);
       }
-      if (j >= 1) {
-        const int pj = j - 1, b = pj & 1, itKp = 2 * pj;
-        ok = mbar_wait_warp(smem_u32(&bars.p_full[b]), (pj >> 1) & 1, abort);
-        if (!ok) break;
-        tc_fence_after_sync();
-        const uint64_t dKp = desc_advance(descRmn, (itKp % NS) * Cfg::kKTileBytes);
-        const uint32_t acc0 = pj > 0 ? 1u : 0u;
-        // dS sits in columns [0,32) of the buffer's S region, P in columns [32,64), packed bf16 pairs
-#pragma unroll
-        for (int kk = 0; kk < kKeys / 16; ++kk) {
-          const uint64_t bd = desc_advance(dKp, kk * 2048);
-          if (elect_one()) umma_ts(tmem + Cfg::kColA, tmem + b * kTile + kk * 8, bd, idesc_a, kk > 0 ? 1u : acc0);
-        }
-#pragma unroll
-        for (int kk = 0; kk < kKeys / 16; ++kk) {
-          const uint64_t bd = desc_advance(dKp, kk * 2048);
-          if (elect_one()) umma_ts(tmem + Cfg::kColM, tmem + b * kTile + 32 + kk * 8, bd, idesc_a, kk > 0 ? 1u : acc0);
-        }
-        if (elect_one()) umma_commit(smem_u32(&bars.kv_empty[itKp % NS]));   // K_{j-1}: S, A and M are done
-        __syncwarp();
+      if (elect_one()) {
+        umma_commit(smem_u32(&bars.s_full[b]));
+        if (which == 1) umma_commit(smem_u32(&bars.kv_empty[it % NS]));   // V_j is used by dP only
       }
+      __syncwarp();
+    }
+  } else if (warp == 3) {
+    // ---------------- A issuer: A += dS K_j ----------------
+    constexpr uint32_t idesc_a = make_idesc_bf16(kTile, D, 0, 1);                  // 128 x D, B = K_j MN-major
+    const uint64_t descRmn = make_smem_desc_sw128(sRing, Cfg::kKSubBytes, 1024);
+    bool ok = true;
+    for (int j = 0; j < n && ok; ++j) {
+      const int b = j & 1, itK = 2 * j;
+      const uint32_t buf = tmem + Cfg::kColBuf + b * 128;
+      ok = mbar_wait_warp(smem_u32(&bars.p_full[b]), (j >> 1) & 1, abort);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint64_t dKj = desc_advance(descRmn, (itK % NS) * Cfg::kKTileBytes);
+      const uint32_t acc0 = j > 0 ? 1u : 0u;
+      // packed dS: keys [0,32) in columns [0,16) of the S region, keys [32,64) in columns [32,48)
+#pragma unroll
+      for (int kk = 0; kk < kKeys / 16; ++kk) {
+        const uint64_t bd = desc_advance(dKj, kk * 2048);
+        if (elect_one()) umma_ts(tmem + Cfg::kColA, buf + (kk >> 1) * 32 + (kk & 1) * 8, bd, idesc_a, kk > 0 ? 1u : acc0);
+      }
+      if (elect_one()) {
+        umma_commit(smem_u32(&bars.kv_empty[itK % NS]));   // K_j: S (before the softmax) and A are done
+        umma_commit(smem_u32(&bars.buf_free[b]));          // tile j+2 may overwrite the buffer
+      }
+      __syncwarp();
     }
     if (ok && elect_one()) umma_commit(smem_u32(&bars.acc_done));
     __syncwarp();
   } else {
-    // ---------------- softmax warpgroups (wg 0: even key tiles, wg 1: odd) + epilogue ----------------
-    const int wg = (warp - 2) >> 2, quad = warp & 3;
+    // ---------------- softmax warps: warpgroup `half` takes key columns [32*half, 32*half+32) ----------------
+    const int half = (warp - 4) >> 2, quad = warp & 3;
     const int row = quad * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const uint32_t S_addr = tmem + lane_addr + wg * kTile;
-    const uint32_t P_addr = S_addr + Cfg::kColP;
     const int qpos = rb.q0 + row;
     const bool live = qpos < rb.q_end;
     const float c = a.scale_log2;
     // rows outside the block get lse = +inf so that P = 0
-    const float2 st = live ? a.stats[(size_t)bh * a.N + qpos] : make_float2(-INFINITY, 0.f);
-    const float nl2 = st.x, Dt = st.y;
-    float Dsum = 0.f, rsum = 0.f;
-    bool ok = true;
-    for (int j = wg; j < n; j += 2) {
-      ok = mbar_wait(smem_u32(&bars.s_full[wg]), (j >> 1) & 1, abort);
+    const float nl2 = live ? a.stats[(size_t)bh * a.N + qpos].x : -INFINITY;
+    const float Dt = live ? a.Dacc[(size_t)bh * a.N + qpos] : 0.f;
+    float rsum = 0.f;
+    // copy this thread's row of Q (warpgroup 0) or dO (warpgroup 1) from the swizzled shared-memory
+    // tile into tensor memory: 16-byte chunk c of row r of a 64-column sub-tile sits at chunk c ^ (r & 7)
+    bool ok = mbar_wait(smem_u32(&bars.q_full), 0, abort);
+    if (ok) {
+      const unsigned char* src = smem_raw + ((half == 0 ? sQ : sdO) - smem_u32(smem_raw)) + row * 128;
+      const uint32_t dst = tmem + lane_addr + (half == 0 ? Cfg::kColQ : Cfg::kColdO);
+#pragma unroll
+      for (int h = 0; h < Cfg::kSub; ++h) {
+        uint32_t v[32];
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          const uint4 x = *reinterpret_cast<const uint4*>(src + h * Cfg::kQSubBytes + ((ch ^ (row & 7)) << 4));
+          v[4 * ch] = x.x; v[4 * ch + 1] = x.y; v[4 * ch + 2] = x.z; v[4 * ch + 3] = x.w;
+        }
+        tmem_st32(dst + h * 32, v);
+      }
+      tmem_wait_st();
+    }
+    tc_fence_before_sync();
+    mbar_arrive(smem_u32(&bars.qt_ready));   // also when the wait gave up: the issuers then see abort
+    for (int j = 0; j < n && ok; ++j) {
+      const int b = j & 1;
+      ok = mbar_wait(smem_u32(&bars.s_full[b]), (j >> 1) & 1, abort);
       if (!ok) break;
       tc_fence_after_sync();
-      uint32_t s[64], dp[64];
-      tmem_ld32(S_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-      tmem_ld32(S_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
-      tmem_ld32(P_addr, *reinterpret_cast<uint32_t(*)[32]>(&dp[0]));
-      tmem_ld32(P_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&dp[32]));
+      const uint32_t S_addr = tmem + lane_addr + Cfg::kColBuf + b * 128 + half * 32;
+      uint32_t s[32], dp[32];
+      tmem_ld32(S_addr, s);
+      tmem_ld32(S_addr + Cfg::kColP, dp);
       tmem_wait_ld();
-      const int limit = j < n_ct ? rb.n_front - j * kKeys : qpos - (rb.dense_start + (j - n_ct) * kKeys) + 1;
-      if (limit < kKeys) {
+      const int limit = (j < n_ct ? rb.n_front - j * kKeys : qpos - (rb.dense_start + (j - n_ct) * kKeys) + 1) - half * 32;
+      if (limit < 32) {
 #pragma unroll
-        for (int i = 0; i < 64; ++i)
+        for (int i = 0; i < 32; ++i)
           if (i >= limit) s[i] = 0xff800000u;
       }
-      uint32_t ds[32], pp[32];
-      float d0 = 0.f, d1 = 0.f, r0 = 0.f, r1 = 0.f;
+      uint32_t ds[16];
+      float r0 = 0.f, r1 = 0.f;
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
+      for (int i = 0; i < 16; ++i) {
         const float p0 = ex2(fmaf(__uint_as_float(s[2 * i]), c, nl2));
         const float p1 = ex2(fmaf(__uint_as_float(s[2 * i + 1]), c, nl2));
-        const float g0 = __uint_as_float(dp[2 * i]), g1 = __uint_as_float(dp[2 * i + 1]);
-        d0 = fmaf(p0, g0, d0);
-        d1 = fmaf(p1, g1, d1);
-        pp[i] = pack_bf16(p0, p1);
-        ds[i] = pack_bf16(p0 * (g0 - Dt), p1 * (g1 - Dt));
+        ds[i] = pack_bf16(p0 * (__uint_as_float(dp[2 * i]) - Dt), p1 * (__uint_as_float(dp[2 * i + 1]) - Dt));
         r0 += __uint_as_float(ds[i] << 16);
         r1 += __uint_as_float(ds[i] & 0xffff0000u);
       }
-      Dsum += d0 + d1;
       rsum += r0 + r1;
-      tmem_st32(S_addr, ds);
-      tmem_st32(S_addr + 32, pp);
+      tmem_st16(S_addr, ds);   // over the first half of this warpgroup's own S columns
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(smem_u32(&bars.p_full[wg]));
+      mbar_arrive(smem_u32(&bars.p_full[b]));
     }
-    red_s[wg][0][row] = Dsum;
-    red_s[wg][1][row] = rsum;
+    red_s[half][row] = rsum;
     asm volatile("bar.sync 1, 256;" ::: "memory");   // the eight softmax warps, whether or not a wait gave up
     if (ok) ok = mbar_wait(smem_u32(&bars.acc_done), 0, abort);
     if (ok) {
       tc_fence_after_sync();
-      const float r = red_s[0][1][row] + red_s[1][1][row];
-      if (wg == 0 && live) a.stats[(size_t)bh * a.N + qpos].y = red_s[0][0][row] + red_s[1][0][row];
+      const float r = red_s[0][row] + red_s[1][row];
       constexpr int CH = D / 2;   // output columns of this warpgroup
-      const uint32_t A_addr = tmem + lane_addr + Cfg::kColA + wg * CH;
-      const uint32_t M_addr = tmem + lane_addr + Cfg::kColM + wg * CH;
-      __nv_bfloat16* orow = a.dQ + ((size_t)bh * a.N + qpos) * D + wg * CH;
+      const uint32_t A_addr = tmem + lane_addr + Cfg::kColA + half * CH;
+      const float* kb = a.kbar + (size_t)bh_kv * D + half * CH;
+      __nv_bfloat16* orow = a.dQ + ((size_t)bh * a.N + qpos) * D + half * CH;
 #pragma unroll
       for (int q = 0; q < CH / 32; ++q) {
-        uint32_t o[32], mk[32];
+        uint32_t o[32];
         tmem_ld32(A_addr + q * 32, o);
-        tmem_ld32(M_addr + q * 32, mk);
         tmem_wait_ld();
         if (live) {
 #pragma unroll
@@ -266,7 +279,7 @@ lrsa_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             float f[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e)
-              f[e] = fmaf(-r, __uint_as_float(mk[8 * v + e]), __uint_as_float(o[8 * v + e])) * a.scale;
+              f[e] = fmaf(-r, __ldg(kb + q * 32 + 8 * v + e), __uint_as_float(o[8 * v + e])) * a.scale;
             uint4 w;
             w.x = pack_bf16(f[0], f[1]); w.y = pack_bf16(f[2], f[3]);
             w.z = pack_bf16(f[4], f[5]); w.w = pack_bf16(f[6], f[7]);
@@ -300,12 +313,47 @@ __global__ void bwd_prep_kernel(const __nv_bfloat16* __restrict__ O, const __nv_
   if (lane == 0) stats[row] = make_float2(-LSE[row] * 1.4426950408889634f, acc);
 }
 
+// kbar[bh][c] += (1/N) * sum of K[bh][t][c] over this block's rows (kbar zeroed beforehand).
+__global__ void __launch_bounds__(256) kbar_kernel(const __nv_bfloat16* __restrict__ K, float* __restrict__ kbar,
+                                                   int N, int d, int rows_per_block) {
+  __shared__ float red[256 * 8];
+  const int bh = blockIdx.y, tid = threadIdx.x;
+  const int lpr = d / 8, rps = 256 / lpr;          // lanes per row (16 bytes each), rows per step
+  const int chunk = tid % lpr, r_in = tid / lpr;
+  const int r0 = blockIdx.x * rows_per_block, r1 = min(N, r0 + rows_per_block);
+  float acc[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+  for (int r = r0 + r_in; r < r1; r += rps) {
+    const uint4 q = *reinterpret_cast<const uint4*>(K + ((size_t)bh * N + r) * d + chunk * 8);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      acc[2 * e] += __uint_as_float(w[e] << 16);
+      acc[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) red[tid * 8 + e] = acc[e];
+  __syncthreads();
+  if (tid < d) {
+    const int ch = tid / 8, e = tid % 8;
+    float sum = 0.f;
+    for (int r = 0; r < rps; ++r) sum += red[(r * lpr + ch) * 8 + e];
+    atomicAdd(kbar + (size_t)bh * d + tid, sum / (float)N);
+  }
+}
+
 }  // namespace
 
 int launch_bwd_prep(const Geom& g, const __nv_bfloat16* O, const __nv_bfloat16* dO, const float* LSE,
-                    float2* stats, cudaStream_t st) {
+                    const __nv_bfloat16* K, float2* stats, float* kbar, cudaStream_t st) {
   const long long rows = (long long)g.B * g.Hq * g.N;
   bwd_prep_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(O, dO, LSE, stats, rows, g.d);
+  LRSA_CUDA_CHECK(cudaGetLastError());
+  launch_counter().n++;
+  const int nsplit = 64, rpb = (g.N + nsplit - 1) / nsplit;
+  kbar_kernel<<<dim3(nsplit, g.B * g.Hkv), 256, 0, st>>>(K, kbar, g.N, g.d, rpb);
   LRSA_CUDA_CHECK(cudaGetLastError());
   launch_counter().n++;
   return LRSA_OK;
@@ -313,8 +361,8 @@ int launch_bwd_prep(const Geom& g, const __nv_bfloat16* O, const __nv_bfloat16* 
 
 template <int D>
 static int launch_dq_t(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO, const __nv_bfloat16* K,
-                       const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, float2* stats,
-                       __nv_bfloat16* dQ, int* status, cudaStream_t st) {
+                       const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, const float2* stats,
+                       const float* Dacc, const float* kbar, __nv_bfloat16* dQ, int* status, cudaStream_t st) {
   using Cfg = DqCfg<D>;
   CUtensorMap mQ, mdO, mK, mV, mKc, mVc;
   const long long rc = g.Rc > 0 ? g.Rc : 1;
@@ -328,7 +376,7 @@ static int launch_dq_t(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat1
   DqArgs a;
   a.plan = make_plan(g, kTile);
   a.BH = g.B * g.Hq; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.N = g.N;
-  a.stats = stats; a.dQ = dQ;
+  a.stats = stats; a.Dacc = Dacc; a.kbar = kbar; a.dQ = dQ;
   a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f;
   a.status = status;
   const long long grid = (long long)a.plan.total * a.BH;
@@ -342,10 +390,10 @@ static int launch_dq_t(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat1
 }
 
 int launch_bwd_dq_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO, const __nv_bfloat16* K,
-                        const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, float2* stats,
-                        __nv_bfloat16* dQ, int* status, cudaStream_t st) {
-  return g.d == 128 ? launch_dq_t<128>(g, Q, dO, K, V, Kc, Vc, stats, dQ, status, st)
-                    : launch_dq_t<64>(g, Q, dO, K, V, Kc, Vc, stats, dQ, status, st);
+                        const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, const float2* stats,
+                        const float* Dacc, const float* kbar, __nv_bfloat16* dQ, int* status, cudaStream_t st) {
+  return g.d == 128 ? launch_dq_t<128>(g, Q, dO, K, V, Kc, Vc, stats, Dacc, kbar, dQ, status, st)
+                    : launch_dq_t<64>(g, Q, dO, K, V, Kc, Vc, stats, Dacc, kbar, dQ, status, st);
 }
 
 }  // namespace lrsa

@@ -5,13 +5,16 @@ namespace lrsa {
 namespace {
 
 struct BwdWs {
-  size_t kc, vc, stats, dkv, total;
+  size_t kbar, dacc, kc, vc, stats, dkv, total;
 };
 BwdWs bwd_ws_layout(const Geom& g) {
   BwdWs w;
   const size_t rc = g.Rc > 0 ? g.Rc : 1;
   const size_t cbytes = align_up((size_t)g.B * g.Hkv * rc * g.d * sizeof(__nv_bfloat16), 1024);
   size_t off = 1024;
+  // cleared together with the header: the mean-key accumulator and the per-row D accumulator
+  w.kbar = off; off += align_up((size_t)g.B * g.Hkv * g.d * sizeof(float), 1024);
+  w.dacc = off; off += align_up((size_t)g.B * g.Hq * g.N * sizeof(float), 1024);
   w.kc = off; off += cbytes;
   w.vc = off; off += cbytes;
   w.stats = off; off += align_up((size_t)g.B * g.Hq * g.N * sizeof(float2), 1024);
@@ -30,17 +33,19 @@ int launch_attn_bwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bflo
                           __nv_bfloat16* dV, void* ws, cudaStream_t st) {
   const BwdWs lay = bwd_ws_layout(g);
   unsigned char* base = static_cast<unsigned char*>(ws);
-  LRSA_CUDA_CHECK(cudaMemsetAsync(base, 0, sizeof(WsHeader), st));
+  LRSA_CUDA_CHECK(cudaMemsetAsync(base, 0, lay.kc, st));
   launch_counter().n++;
   __nv_bfloat16* Kc = reinterpret_cast<__nv_bfloat16*>(base + lay.kc);
   __nv_bfloat16* Vc = reinterpret_cast<__nv_bfloat16*>(base + lay.vc);
   float2* stats = reinterpret_cast<float2*>(base + lay.stats);
+  float* kbar = reinterpret_cast<float*>(base + lay.kbar);
+  float* Dacc = reinterpret_cast<float*>(base + lay.dacc);
   int* status = &reinterpret_cast<WsHeader*>(base)->status;
   int rc = launch_compact_kv(g, K, V, idx, Kc, Vc, st);
-  if (rc == LRSA_OK) rc = launch_bwd_prep(g, O, dO, LSE, stats, st);
-  if (rc == LRSA_OK) rc = launch_bwd_dq_sm100(g, Q, dO, K, V, Kc, Vc, stats, dQ, status, st);
+  if (rc == LRSA_OK) rc = launch_bwd_prep(g, O, dO, LSE, K, stats, kbar, st);
   if (rc == LRSA_OK)
-    rc = launch_bwd_dkv_sm100(g, Q, dO, K, V, Kc, Vc, stats, idx, dK, dV, base + lay.dkv, status, st);
+    rc = launch_bwd_dkv_sm100(g, Q, dO, K, V, Kc, Vc, stats, Dacc, idx, dK, dV, base + lay.dkv, status, st);
+  if (rc == LRSA_OK) rc = launch_bwd_dq_sm100(g, Q, dO, K, V, Kc, Vc, stats, Dacc, kbar, dQ, status, st);
   return rc;
 }
 

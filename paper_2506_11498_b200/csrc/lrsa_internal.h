@@ -86,18 +86,19 @@ int launch_attn_bwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bflo
                           const __nv_bfloat16* V, const __nv_bfloat16* O, const __nv_bfloat16* dO,
                           const float* LSE, const int32_t* idx, __nv_bfloat16* dQ, __nv_bfloat16* dK,
                           __nv_bfloat16* dV, void* ws, cudaStream_t st);
-// stats[row] = (-LSE * log2(e), rowsum(dO * O)) per query row.  The dQ kernel replaces the second
-// component by the accurate sum_j P dP it accumulates; the dK/dV kernel runs after it and reads that.
+// Backward helpers.  stats[row] = (-LSE * log2(e), rowsum(dO * O)) per query row; kbar[b*Hkv+h][c] is the
+// mean key (accumulated into a zeroed array).  The dK/dV kernel runs first and adds sum_j P dP, the
+// accurate D of every query row, into the zeroed Dacc; the dQ kernel reads it.
 int launch_bwd_prep(const Geom& g, const __nv_bfloat16* O, const __nv_bfloat16* dO, const float* LSE,
-                    float2* stats, cudaStream_t st);
+                    const __nv_bfloat16* K, float2* stats, float* kbar, cudaStream_t st);
 int launch_bwd_dq_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO, const __nv_bfloat16* K,
-                        const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, float2* stats,
-                        __nv_bfloat16* dQ, int* status, cudaStream_t st);
+                        const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, const float2* stats,
+                        const float* Dacc, const float* kbar, __nv_bfloat16* dQ, int* status, cudaStream_t st);
 
 size_t dkv_ws_bytes(const Geom& g, size_t* prefix_bytes);
 int launch_bwd_dkv_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO, const __nv_bfloat16* K,
                          const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, const float2* stats,
-                         const int32_t* idx, __nv_bfloat16* dK, __nv_bfloat16* dV, void* ws_dkv,
+                         float* Dacc, const int32_t* idx, __nv_bfloat16* dK, __nv_bfloat16* dV, void* ws_dkv,
                          int* status, cudaStream_t st);
 
 #define LRSA_CUDA_CHECK(expr)                                 \
