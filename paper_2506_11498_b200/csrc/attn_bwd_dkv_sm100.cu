@@ -12,7 +12,11 @@
 //   dV  += P^T dO_i      (TMEM x smem -> TMEM)
 //   dK  += dS^T Q_i      (TMEM x smem -> TMEM)
 // P^T and dS^T are written back over S^T and dP^T as packed bf16; both are double-buffered so the
-// tensor core computes the next S^T/dP^T while one warpgroup handles the current pair.  At the end
+// tensor core computes the next S^T/dP^T while the current pair is in the softmax, on which both
+// warpgroups work (32 query columns each).  Warps: 0 producer, 1-3 tensor-core issuers (S^T, dP^T,
+// dV/dK), 4-11 softmax and epilogue.  The softmax warps also sum P^T * dP^T over the keys and add it to
+// a per-query-row accumulator: D_i = sum_j P_ij dP_ij, the accurate replacement of rowsum(dO * O)
+// that the dQ kernel (which runs afterwards) needs.  At the end
 // the accumulators are added (fp32 atomics) to a zeroed workspace indexed by original position
 // (dense tiles) or by compact row (compact tiles); two small kernels then fold the compact rows
 // onto their original positions and convert to bf16.
@@ -117,7 +121,7 @@ struct DkvCfg {
   static constexpr int kStageBytes = 2 * kQTileBytes;       // Q_i + dO_i
   static constexpr int kStages = D == 128 ? 4 : 8;
   static constexpr int kSmem = 2 * kKTileBytes + kStages * kStageBytes + 1024;
-  static constexpr int kThreads = 320;
+  static constexpr int kThreads = 384;   // producer, three MMA issuers, eight softmax warps
   static constexpr uint32_t kColS = 0, kColP = 128, kColK = 256, kColV = 256 + D;
 };
 
@@ -137,7 +141,7 @@ struct DkvArgs {
 struct DkvBars {
   uint64_t kv_full, acc_done;
   uint64_t ring_full[8], ring_empty[8];
-  uint64_t s_full[2], p_full[2];
+  uint64_t s_full[2], p_full[2], buf_free[2];
 };
 
 __device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
@@ -181,7 +185,11 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     mbar_init(smem_u32(&bars.kv_full), 1);
     mbar_init(smem_u32(&bars.acc_done), 1);
     for (int i = 0; i < NS; ++i) { mbar_init(smem_u32(&bars.ring_full[i]), 1); mbar_init(smem_u32(&bars.ring_empty[i]), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&bars.s_full[b]), 1); mbar_init(smem_u32(&bars.p_full[b]), 128); }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars.s_full[b]), 2);      // the S^T issuer and the dP^T issuer
+      mbar_init(smem_u32(&bars.p_full[b]), 256);    // every softmax thread
+      mbar_init(smem_u32(&bars.buf_free[b]), 1);
+    }
     fence_barrier_init();
   }
   if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_s), 512); tmem_relinquish(); }
@@ -250,86 +258,88 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         while (!mbar_try_wait(smem_u32(&bars.ring_full[i2 % NS]), (i2 / NS) & 1) && clock64() - t0 < 2000000) {}
       }
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer: the whole warp runs the loop, one elected lane issues ----------------
-    constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kQRows, 0, 0);  // S^T, dP^T : 128 keys x 64 queries
-    constexpr uint32_t idesc_a = make_idesc_bf16(kTile, D, 0, 1);       // dV, dK    : 128 keys x D
-    const uint64_t descK = make_smem_desc_sw128(sK, 16, 1024), descV = make_smem_desc_sw128(sV, 16, 1024);
-    const uint64_t descR = make_smem_desc_sw128(sRing, 16, 1024);                    // K-major Q_i / dO_i
-    const uint64_t descRmn = make_smem_desc_sw128(sRing, Cfg::kQSubBytes, 1024);     // MN-major Q_i / dO_i
+  } else if (warp == 1 || warp == 2) {
+    // ---------------- S^T issuer (warp 1: K_j Q_i^T) and dP^T issuer (warp 2: V_j dO_i^T) ----------------
+    // Each issuing warp runs its loop with all lanes (uniform control flow, descriptors computed once)
+    // and elects one lane per instruction.
+    const int which = warp - 1;
+    constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kQRows, 0, 0);  // 128 keys x 64 queries
+    const uint64_t descA = make_smem_desc_sw128(which == 0 ? sK : sV, 16, 1024);
+    const uint64_t descR = make_smem_desc_sw128(sRing + which * Cfg::kQTileBytes, 16, 1024);   // K-major Q_i / dO_i
     bool ok = mbar_wait_warp(smem_u32(&bars.kv_full), 0, abort);
-    for (int it = 0; it <= n && ok; ++it) {
-      if (it < n) {
-        const int slot = it % NS, b = it & 1;
-        ok = mbar_wait_warp(smem_u32(&bars.ring_full[slot]), (it / NS) & 1, abort);
-        if (!ok) break;
-        tc_fence_after_sync();
-        const uint64_t dQi = desc_advance(descR, slot * Cfg::kStageBytes);
-        const uint64_t ddOi = desc_advance(dQi, Cfg::kQTileBytes);
+    for (int it = 0; it < n && ok; ++it) {
+      const int slot = it % NS, b = it & 1;
+      ok = mbar_wait_warp(smem_u32(&bars.ring_full[slot]), (it / NS) & 1, abort);
+      if (ok && it >= 2) ok = mbar_wait_warp(smem_u32(&bars.buf_free[b]), ((it >> 1) - 1) & 1, abort);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t d_tmem = tmem + (which == 0 ? Cfg::kColS : Cfg::kColP) + b * kQRows;
+      const uint64_t dB = desc_advance(descR, slot * Cfg::kStageBytes);
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t koff = (kk >> 2) * Cfg::kKSubBytes + (kk & 3) * 32;
-          const uint32_t qoff = (kk >> 2) * Cfg::kQSubBytes + (kk & 3) * 32;
-          const uint64_t ad = desc_advance(descK, koff), bd = desc_advance(dQi, qoff);
-          if (elect_one()) umma_ss(tmem + Cfg::kColS + b * kQRows, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
-        }
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t koff = (kk >> 2) * Cfg::kKSubBytes + (kk & 3) * 32;
-          const uint32_t qoff = (kk >> 2) * Cfg::kQSubBytes + (kk & 3) * 32;
-          const uint64_t ad = desc_advance(descV, koff), bd = desc_advance(ddOi, qoff);
-          if (elect_one()) umma_ss(tmem + Cfg::kColP + b * kQRows, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
-        }
-        if (elect_one()) umma_commit(smem_u32(&bars.s_full[b]));
-        __syncwarp();
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const uint32_t koff = (kk >> 2) * Cfg::kKSubBytes + (kk & 3) * 32;
+        const uint32_t qoff = (kk >> 2) * Cfg::kQSubBytes + (kk & 3) * 32;
+        const uint64_t ad = desc_advance(descA, koff), bd = desc_advance(dB, qoff);
+        if (elect_one()) umma_ss(d_tmem, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
       }
-      if (it >= 1) {
-        const int pi = it - 1, slot = pi % NS, b = pi & 1;
-        ok = mbar_wait_warp(smem_u32(&bars.p_full[b]), (pi >> 1) & 1, abort);
-        if (!ok) break;
-        tc_fence_after_sync();
-        const uint64_t dQi = desc_advance(descRmn, slot * Cfg::kStageBytes);
-        const uint64_t ddOi = desc_advance(dQi, Cfg::kQTileBytes);
-        const uint32_t acc0 = pi > 0 ? 1u : 0u;
+      if (elect_one()) umma_commit(smem_u32(&bars.s_full[b]));
+      __syncwarp();
+    }
+  } else if (warp == 3) {
+    // ---------------- dV / dK issuer ----------------
+    constexpr uint32_t idesc_a = make_idesc_bf16(kTile, D, 0, 1);       // 128 keys x D
+    const uint64_t descRmn = make_smem_desc_sw128(sRing, Cfg::kQSubBytes, 1024);     // MN-major Q_i / dO_i
+    bool ok = true;
+    for (int it = 0; it < n && ok; ++it) {
+      const int slot = it % NS, b = it & 1;
+      ok = mbar_wait_warp(smem_u32(&bars.p_full[b]), (it >> 1) & 1, abort);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint64_t dQi = desc_advance(descRmn, slot * Cfg::kStageBytes);
+      const uint64_t ddOi = desc_advance(dQi, Cfg::kQTileBytes);
+      const uint32_t acc0 = it > 0 ? 1u : 0u;
+      // packed P^T / dS^T: queries [0,32) in columns [0,16) of the buffer, queries [32,64) in columns [32,48)
 #pragma unroll
-        for (int kk = 0; kk < kQRows / 16; ++kk) {
-          const uint64_t bd = desc_advance(ddOi, kk * 2048);
-          if (elect_one())
-            umma_ts(tmem + Cfg::kColV, tmem + Cfg::kColS + b * kQRows + kk * 8, bd, idesc_a, kk > 0 ? 1u : acc0);
-        }
-#pragma unroll
-        for (int kk = 0; kk < kQRows / 16; ++kk) {
-          const uint64_t bd = desc_advance(dQi, kk * 2048);
-          if (elect_one())
-            umma_ts(tmem + Cfg::kColK, tmem + Cfg::kColP + b * kQRows + kk * 8, bd, idesc_a, kk > 0 ? 1u : acc0);
-        }
-        if (elect_one()) umma_commit(smem_u32(&bars.ring_empty[slot]));
-        __syncwarp();
+      for (int kk = 0; kk < kQRows / 16; ++kk) {
+        const uint64_t bd = desc_advance(ddOi, kk * 2048);
+        if (elect_one())
+          umma_ts(tmem + Cfg::kColV, tmem + Cfg::kColS + b * kQRows + (kk >> 1) * 32 + (kk & 1) * 8, bd, idesc_a,
+                  kk > 0 ? 1u : acc0);
       }
+#pragma unroll
+      for (int kk = 0; kk < kQRows / 16; ++kk) {
+        const uint64_t bd = desc_advance(dQi, kk * 2048);
+        if (elect_one())
+          umma_ts(tmem + Cfg::kColK, tmem + Cfg::kColP + b * kQRows + (kk >> 1) * 32 + (kk & 1) * 8, bd, idesc_a,
+                  kk > 0 ? 1u : acc0);
+      }
+      if (elect_one()) {
+        umma_commit(smem_u32(&bars.ring_empty[slot]));
+        umma_commit(smem_u32(&bars.buf_free[b]));      // tile it+2 may overwrite the buffer
+      }
+      __syncwarp();
     }
     if (ok && elect_one()) umma_commit(smem_u32(&bars.acc_done));
     __syncwarp();
   } else {
-    // ---------------- P^T / dS^T warpgroups + epilogue ----------------
-    const int wg = (warp - 2) >> 2, quad = warp & 3;
+    // ---------------- P^T / dS^T: warpgroup `wg` takes query columns [32*wg, 32*wg+32) of every tile ----------------
+    const int wg = (warp - 4) >> 2, quad = warp & 3;
     const int r = quad * 32 + lane;            // key row of this thread inside the tile
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const float c = a.scale_log2;
     const bool key_ok = kt.row0 + r < kt.key_end;
     bool ok = true;
-    for (int it = wg; it < n; it += 2) {
-      const int slot = it % NS;
-      ok = mbar_wait(smem_u32(&bars.s_full[wg]), (it >> 1) & 1, abort);
+    for (int it = 0; it < n; ++it) {
+      const int slot = it % NS, b = it & 1;
+      ok = mbar_wait(smem_u32(&bars.s_full[b]), (it >> 1) & 1, abort);
       if (ok) ok = mbar_wait(smem_u32(&bars.ring_full[slot]), (it / NS) & 1, abort);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t S_addr = tmem + lane_addr + Cfg::kColS + wg * kQRows;
-      const uint32_t P_addr = tmem + lane_addr + Cfg::kColP + wg * kQRows;
-      uint32_t s[64], dp[64];
-      tmem_ld32(S_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-      tmem_ld32(S_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
-      tmem_ld32(P_addr, *reinterpret_cast<uint32_t(*)[32]>(&dp[0]));
-      tmem_ld32(P_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&dp[32]));
+      const uint32_t S_addr = tmem + lane_addr + Cfg::kColS + b * kQRows + wg * 32;
+      const uint32_t P_addr = tmem + lane_addr + Cfg::kColP + b * kQRows + wg * 32;
+      uint32_t s[32], dp[32];
+      tmem_ld32(S_addr, s);
+      tmem_ld32(P_addr, dp);
       tmem_wait_ld();
       // first query column of this tile that sees this thread's key (64 = none)
       const int gi = it_begin + it;
@@ -349,17 +359,18 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
           col = p.S + (cch + 1) * p.L - q0;         // first column of the next chunk
         }
       }
+      lo -= wg * 32;
       if (lo > 0) {
 #pragma unroll
-        for (int i = 0; i < 64; ++i)
+        for (int i = 0; i < 32; ++i)
           if (i < lo) s[i] = 0xff800000u;
       }
-      const float4* nl2v = reinterpret_cast<const float4*>(st_nl2[slot]);
-      const float4* Dv = reinterpret_cast<const float4*>(st_D[slot]);
-      uint32_t pp[32], ds[32];
-      float x[64];   // P * dP, whose sum over the keys is the accurate D of the query column
+      const float4* nl2v = reinterpret_cast<const float4*>(st_nl2[slot] + wg * 32);
+      const float4* Dv = reinterpret_cast<const float4*>(st_D[slot] + wg * 32);
+      uint32_t pp[16], ds[16];
+      float x[32];   // P * dP, whose sum over the keys is the accurate D of the query column
 #pragma unroll
-      for (int v = 0; v < 16; ++v) {
+      for (int v = 0; v < 8; ++v) {
         const float4 nl = nl2v[v], dd = Dv[v];
         const float p0 = ex2(fmaf(__uint_as_float(s[4 * v + 0]), c, nl.x));
         const float p1 = ex2(fmaf(__uint_as_float(s[4 * v + 1]), c, nl.y));
@@ -373,15 +384,15 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         ds[2 * v + 1] = pack_bf16(p2 * (g2 - dd.z), p3 * (g3 - dd.w));
         x[4 * v + 0] = p0 * g0; x[4 * v + 1] = p1 * g1; x[4 * v + 2] = p2 * g2; x[4 * v + 3] = p3 * g3;
       }
-      tmem_st32(S_addr, pp);
-      tmem_st32(P_addr, ds);
+      tmem_st16(S_addr, pp);   // over the first half of this warpgroup's own columns
+      tmem_st16(P_addr, ds);
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(smem_u32(&bars.p_full[wg]));
+      mbar_arrive(smem_u32(&bars.p_full[b]));
       // Off the tensor core's critical path: sum x over the warp's 32 keys by halving exchanges; lane l
-      // ends with query columns 2l and 2l+1, which it adds to the per-row accumulator in global memory.
+      // ends with query column 32*wg + l, which it adds to the per-row accumulator in global memory.
 #pragma unroll
-      for (int m = 32, bit = 16; m >= 2; m >>= 1, bit >>= 1) {
+      for (int m = 16, bit = 16; m >= 1; m >>= 1, bit >>= 1) {
         const bool up = (lane & bit) != 0;
 #pragma unroll
         for (int i = 0; i < m; ++i) {
@@ -391,10 +402,8 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         }
       }
       {
-        const int hq = hq0 + gi / kt.nq;
-        float* drow = a.Dacc + (size_t)hq * p.N + q0 + 2 * lane;
-        if (q0 + 2 * lane < kt.qend) atomicAdd(drow, x[0]);
-        if (q0 + 2 * lane + 1 < kt.qend) atomicAdd(drow + 1, x[1]);
+        const int hq = hq0 + gi / kt.nq, q = q0 + wg * 32 + lane;
+        if (q < kt.qend) atomicAdd(a.Dacc + (size_t)hq * p.N + q, x[0]);
       }
     }
     if (ok) ok = mbar_wait(smem_u32(&bars.acc_done), 0, abort);
