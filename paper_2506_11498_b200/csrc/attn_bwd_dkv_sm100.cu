@@ -160,6 +160,8 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
   __shared__ __align__(8) DkvBars bars;
   __shared__ __align__(16) float st_nl2[NS][kQRows];   // -LSE*log2(e) per query row of the stage (-inf: not seen)
   __shared__ __align__(16) float st_D[NS][kQRows];
+  __shared__ int st_meta[NS][4];             // compact tiles: compact rows visible to the stage's first chunk,
+                                             // first column of its second chunk, rows visible to that chunk
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
 
@@ -239,6 +241,12 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         st_nl2[slot][lane + 32 * k] = cur[k].x;
         st_D[slot][lane + 32 * k] = cur[k].y;
         cur[k] = nxt[k];
+      }
+      if (lane == 0 && kt.kind == 0) {
+        const int cch = (q0 - p.S) / p.L;
+        st_meta[slot][0] = p.S + n_hist_windows(cch, p.ndp, p.Wsel) * p.K;
+        st_meta[slot][1] = min(kQRows, p.S + (cch + 1) * p.L - q0);
+        st_meta[slot][2] = p.S + n_hist_windows(cch + 1, p.ndp, p.Wsel) * p.K;
       }
       __syncwarp();
       if (lane == 0) {
@@ -349,6 +357,9 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         lo = kQRows;
       } else if (kt.kind == 1) {
         lo = kt.row0 + r - q0;                      // causal: query position >= key position
+      } else if (p.L >= kQRows) {                   // compact row, tile spans at most two chunks
+        const int cr = kt.row0 + r;
+        lo = cr < st_meta[slot][0] ? 0 : (cr < st_meta[slot][2] ? st_meta[slot][1] : kQRows);
       } else {
         const int cr = kt.row0 + r;                 // compact row: needs cr < S + n_hist(chunk)*K
         lo = kQRows;
@@ -380,17 +391,18 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         const float g2 = __uint_as_float(dp[4 * v + 2]), g3 = __uint_as_float(dp[4 * v + 3]);
         pp[2 * v] = pack_bf16(p0, p1);
         pp[2 * v + 1] = pack_bf16(p2, p3);
-        ds[2 * v] = pack_bf16(p0 * (g0 - dd.x), p1 * (g1 - dd.y));
-        ds[2 * v + 1] = pack_bf16(p2 * (g2 - dd.z), p3 * (g3 - dd.w));
         x[4 * v + 0] = p0 * g0; x[4 * v + 1] = p1 * g1; x[4 * v + 2] = p2 * g2; x[4 * v + 3] = p3 * g3;
+        ds[2 * v] = pack_bf16(fmaf(-p0, dd.x, x[4 * v + 0]), fmaf(-p1, dd.y, x[4 * v + 1]));
+        ds[2 * v + 1] = pack_bf16(fmaf(-p2, dd.z, x[4 * v + 2]), fmaf(-p3, dd.w, x[4 * v + 3]));
       }
       tmem_st16(S_addr, pp);   // over the first half of this warpgroup's own columns
       tmem_st16(P_addr, ds);
       tmem_wait_st();
       tc_fence_before_sync();
       mbar_arrive(smem_u32(&bars.p_full[b]));
-      // Off the tensor core's critical path: sum x over the warp's 32 keys by halving exchanges; lane l
-      // ends with query column 32*wg + l, which it adds to the per-row accumulator in global memory.
+      // Off the tensor core's critical path: sum x over the warp's 32 keys by halving exchanges (register
+      // shuffles: shared-memory bandwidth is what the tensor core's operands need); lane l ends with
+      // query column 32*wg + l, which it adds to the per-row accumulator in global memory.
 #pragma unroll
       for (int m = 16, bit = 16; m >= 1; m >>= 1, bit >>= 1) {
         const bool up = (lane & bit) != 0;

@@ -1,17 +1,19 @@
 // LRSA attention forward on tcgen05 tensor cores (Section 3.1 Eq. 3 under the chunked mask of
 // Section 3.2).
 //
-// A CTA owns a block of 256 query rows of one (batch, query head): two 128-row tiles that share one
-// key list (first n_front rows of the compact sinks+kept buffer, then a contiguous range of original
-// positions up to the diagonal).  Roles:
-//   warp 0      TMA producer: Q tiles once, then K_j, V_j tiles through a ring of shared-memory slots
-//   warp 1      MMA issuer:  S_t = Q_t K_j^T (operands in shared memory) and O_t += P_t V_j with P_t
-//               read from tensor memory; owns the TMEM allocation
-//   warps 2-5   softmax of tile 0, warps 6-9 softmax of tile 1: S from TMEM, online softmax in fp32
-//               with the maximum only raised when it grew by more than 2^8 (then O is rescaled in
-//               TMEM), P written back over S as packed bf16
-// While one tile's softmax runs, the tensor core works on the other tile.  All mbarrier waits are
-// bounded; on expiry the CTA records LRSA_ERR_TIMEOUT in the workspace header and leaves.
+// A CTA owns one 128-row query tile of one (batch, query head) and walks its key list (first n_front
+// rows of the compact sinks+kept buffer, then a contiguous range of original positions up to the
+// diagonal) in 128-key tiles.  Q is copied once into tensor memory, so both products take their
+// 128-row operand from TMEM and only K_j / V_j from shared memory.  Roles:
+//   warp 0      TMA producer: the Q tile once, then K_j, V_j tiles through a ring of shared-memory slots
+//   warp 1      issues S_j = Q K_j^T into one of two TMEM buffers; owns the TMEM allocation
+//   warp 2      issues O += P_j V_j with P_j read from tensor memory
+//   warps 4-11  softmax: both warpgroups work on every tile, 64 key columns each; S from TMEM, online
+//               softmax in fp32 with the maximum only raised when it grew by more than 2^8 (then O is
+//               rescaled in TMEM), P written back over S as packed bf16
+// S is double-buffered, so the tensor core computes S_{j+1} while tile j is in the softmax.  The
+// issuing warps run their loops with all lanes and elect one lane per instruction.  All mbarrier
+// waits are bounded; on expiry the CTA records LRSA_ERR_TIMEOUT in the workspace header and leaves.
 #include "attn_common_sm100.h"
 
 namespace lrsa {
@@ -24,10 +26,11 @@ struct FwdCfg {
   static constexpr int kSub = D / 64;                 // 64-column (128-byte) sub-tiles per tile
   static constexpr int kSubBytes = kTile * 128;       // 16 KB
   static constexpr int kTileBytes = kSub * kSubBytes; // one Q / K / V tile
-  static constexpr int kStages = D == 128 ? 5 : 8;    // K/V ring slots
-  static constexpr int kSmem = (2 + kStages) * kTileBytes + 1024;
-  static constexpr int kThreads = 320;
-  static constexpr uint32_t kColS = 0, kColO = 256;   // TMEM columns: S0,S1 then O0,O1
+  static constexpr int kStages = D == 128 ? 6 : 12;   // K/V ring slots
+  static constexpr int kSmem = (1 + kStages) * kTileBytes + 1024;
+  static constexpr int kThreads = 384;
+  // TMEM columns: Q as packed bf16 (D/2 columns), the accumulator O at 64, S buffer b at 256 + 128b
+  static constexpr uint32_t kColQ = 0, kColO = 64, kColS = 256;
 };
 
 struct FwdArgs {
@@ -40,9 +43,9 @@ struct FwdArgs {
 };
 
 struct FwdBars {
-  uint64_t q_full;
-  uint64_t kv_full[8], kv_empty[8];
-  uint64_t s_full[2], p_full[2], pv_done[2];
+  uint64_t q_full, qt_ready, pv_done;
+  uint64_t kv_full[12], kv_empty[12];
+  uint64_t s_full[2], p_full[2], buf_free[2];
 };
 
 template <int D>
@@ -54,33 +57,30 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   constexpr int NS = Cfg::kStages;
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) FwdBars bars;
+  __shared__ float red_s[2][kTile];   // [column half][row] partial row sums
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sQ = smem0, sRing = smem0 + 2 * Cfg::kTileBytes;
+  const uint32_t sQ = smem0, sRing = smem0 + Cfg::kTileBytes;
 
   const int bh = blockIdx.x % a.BH, blk = blockIdx.x / a.BH;
   const RowBlock rb = decode_block(a.plan, blk);
   const int bh_kv = (bh / a.Hq) * a.Hkv + (bh % a.Hq) / a.G;
   const int n_ct = (rb.n_front + kTile - 1) / kTile;
-  int n_t[2];
-#pragma unroll
-  for (int t = 0; t < 2; ++t) {
-    const int first = rb.q0 + t * kTile;
-    n_t[t] = first >= rb.q_end ? 0 : n_ct + (min(first + kTile - 1, rb.q_end - 1) - rb.dense_start) / kTile + 1;
-  }
-  const int n_max = max(n_t[0], n_t[1]);
+  const int n = n_ct + (rb.q_end - 1 - rb.dense_start) / kTile + 1;   // key tiles of this block (>= 1)
 
   if (tid == 0) {
     abort_s = 0;
     mbar_init(smem_u32(&bars.q_full), 1);
+    mbar_init(smem_u32(&bars.qt_ready), 256);
+    mbar_init(smem_u32(&bars.pv_done), 1);
     for (int i = 0; i < NS; ++i) { mbar_init(smem_u32(&bars.kv_full[i]), 1); mbar_init(smem_u32(&bars.kv_empty[i]), 1); }
-    for (int t = 0; t < 2; ++t) {
-      mbar_init(smem_u32(&bars.s_full[t]), 1);
-      mbar_init(smem_u32(&bars.p_full[t]), 128);
-      mbar_init(smem_u32(&bars.pv_done[t]), 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars.s_full[b]), 1);
+      mbar_init(smem_u32(&bars.p_full[b]), 256);    // every softmax thread
+      mbar_init(smem_u32(&bars.buf_free[b]), 1);
     }
     fence_barrier_init();
   }
@@ -96,14 +96,12 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     if (lane == 0) {
       prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV);
       prefetch_tensormap(&mapKc); prefetch_tensormap(&mapVc);
-      mbar_expect_tx(smem_u32(&bars.q_full), 2 * Cfg::kTileBytes);
-      for (int t = 0; t < 2; ++t)
-        for (int h = 0; h < Cfg::kSub; ++h)
-          tma_load_3d(sQ + t * Cfg::kTileBytes + h * Cfg::kSubBytes, &mapQ, h * 64, rb.q0 + t * kTile, bh,
-                      smem_u32(&bars.q_full));
+      mbar_expect_tx(smem_u32(&bars.q_full), Cfg::kTileBytes);
+      for (int h = 0; h < Cfg::kSub; ++h)
+        tma_load_3d(sQ + h * Cfg::kSubBytes, &mapQ, h * 64, rb.q0, bh, smem_u32(&bars.q_full));
       int it = 0;
       bool ok = true;
-      for (int j = 0; j < n_max && ok; ++j) {
+      for (int j = 0; j < n && ok; ++j) {
         for (int which = 0; which < 2 && ok; ++which, ++it) {
           const int slot = it % NS, use = it / NS;
           if (use > 0) ok = mbar_wait(smem_u32(&bars.kv_empty[slot]), (use - 1) & 1, abort);
@@ -127,97 +125,132 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer: the whole warp runs the loop, one elected lane issues ----------------
+    // ---------------- S issuer: S_j = Q K_j^T into buffer j & 1 ----------------
     constexpr uint32_t idesc_qk = make_idesc_bf16(kTile, kTile, 0, 0);
-    constexpr uint32_t idesc_pv = make_idesc_bf16(kTile, D, 0, 1);
-    const uint64_t descQ = make_smem_desc_sw128(sQ, 16, 1024);
     const uint64_t descK0 = make_smem_desc_sw128(sRing, 16, 1024);
-    const uint64_t descV0 = make_smem_desc_sw128(sRing, Cfg::kSubBytes, 1024);
-    bool ok = mbar_wait_warp(smem_u32(&bars.q_full), 0, abort);
-    for (int j = 0; j <= n_max && ok; ++j) {
-      const int itK = 2 * j, itV = 2 * j - 1;
-      if (j < n_max) ok = mbar_wait_warp(smem_u32(&bars.kv_full[itK % NS]), (itK / NS) & 1, abort);
-      if (ok && j >= 1) ok = mbar_wait_warp(smem_u32(&bars.kv_full[itV % NS]), (itV / NS) & 1, abort);
+    bool ok = mbar_wait_warp(smem_u32(&bars.qt_ready), 0, abort);   // Q is in tensor memory
+    for (int j = 0; j < n && ok; ++j) {
+      const int it = 2 * j, b = j & 1;   // ring order: K_j at 2j, V_j at 2j+1
+      ok = mbar_wait_warp(smem_u32(&bars.kv_full[it % NS]), (it / NS) & 1, abort);
+      if (ok && j >= 2) ok = mbar_wait_warp(smem_u32(&bars.buf_free[b]), ((j >> 1) - 1) & 1, abort);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint64_t dK = desc_advance(descK0, (itK % NS) * Cfg::kTileBytes);
-      const uint64_t dV = desc_advance(descV0, ((itV + NS) % NS) * Cfg::kTileBytes);
+      const uint64_t dK = desc_advance(descK0, (it % NS) * Cfg::kTileBytes);
 #pragma unroll
-      for (int t = 0; t < 2; ++t) {
-        const bool do_qk = j < n_t[t], do_pv = j >= 1 && (j - 1) < n_t[t];
-        if (do_pv && ok) {
-          ok = mbar_wait_warp(smem_u32(&bars.p_full[t]), (j - 1) & 1, abort);
-          if (ok) {
-            tc_fence_after_sync();
-            const uint32_t acc0 = j - 1 > 0 ? 1u : 0u;
-#pragma unroll
-            for (int kk = 0; kk < kTile / 16; ++kk) {
-              const uint64_t bd = desc_advance(dV, kk * 2048);
-              if (elect_one())
-                umma_ts(tmem + Cfg::kColO + t * D, tmem + Cfg::kColS + t * kTile + kk * 8, bd, idesc_pv,
-                        kk > 0 ? 1u : acc0);
-            }
-            if (elect_one()) umma_commit(smem_u32(&bars.pv_done[t]));
-            __syncwarp();
-          }
-        }
-        if (do_qk && ok) {
-#pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t off = (kk >> 2) * Cfg::kSubBytes + (kk & 3) * 32;
-            const uint64_t ad = desc_advance(descQ, t * Cfg::kTileBytes + off), bd = desc_advance(dK, off);
-            if (elect_one()) umma_ss(tmem + Cfg::kColS + t * kTile, ad, bd, idesc_qk, kk > 0 ? 1u : 0u);
-          }
-          if (elect_one()) umma_commit(smem_u32(&bars.s_full[t]));
-          __syncwarp();
-        }
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const uint64_t bd = desc_advance(dK, (kk >> 2) * Cfg::kSubBytes + (kk & 3) * 32);
+        if (elect_one()) umma_ts(tmem + Cfg::kColS + b * kTile, tmem + Cfg::kColQ + kk * 8, bd, idesc_qk, kk > 0 ? 1u : 0u);
       }
-      if (!ok) break;
-      if (j < n_max && elect_one()) umma_commit(smem_u32(&bars.kv_empty[itK % NS]));
-      __syncwarp();
-      if (j >= 1 && elect_one()) umma_commit(smem_u32(&bars.kv_empty[itV % NS]));
+      if (elect_one()) {
+        umma_commit(smem_u32(&bars.s_full[b]));
+        umma_commit(smem_u32(&bars.kv_empty[it % NS]));   // K_j is used by S_j only
+      }
       __syncwarp();
     }
-  } else {
-    // ---------------- softmax + epilogue ----------------
-    const int t = (warp - 2) >> 2, quad = warp & 3;
-    const int row = quad * 32 + lane;
-    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const uint32_t S_addr = tmem + lane_addr + Cfg::kColS + t * kTile;
-    const uint32_t O_addr = tmem + lane_addr + Cfg::kColO + t * D;
-    const int qpos = rb.q0 + t * kTile + row;
-    const int n = n_t[t];
-    const float c = a.scale_log2;
-    float m = -INFINITY, l = 0.f;
+  } else if (warp == 2) {
+    // ---------------- O issuer: O += P_j V_j ----------------
+    constexpr uint32_t idesc_pv = make_idesc_bf16(kTile, D, 0, 1);
+    const uint64_t descV0 = make_smem_desc_sw128(sRing, Cfg::kSubBytes, 1024);   // V_j MN-major
     bool ok = true;
-    for (int j = 0; j < n; ++j) {
-      ok = mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort);
+    for (int j = 0; j < n && ok; ++j) {
+      const int it = 2 * j + 1, b = j & 1;
+      ok = mbar_wait_warp(smem_u32(&bars.kv_full[it % NS]), (it / NS) & 1, abort);
+      if (ok) ok = mbar_wait_warp(smem_u32(&bars.p_full[b]), (j >> 1) & 1, abort);
       if (!ok) break;
       tc_fence_after_sync();
-      uint32_t s[128];
+      const uint64_t dV = desc_advance(descV0, (it % NS) * Cfg::kTileBytes);
+      const uint32_t acc0 = j > 0 ? 1u : 0u;
+      // packed P: keys [0,64) in columns [0,32) of the buffer, keys [64,128) in columns [64,96)
 #pragma unroll
-      for (int q = 0; q < 4; ++q) tmem_ld32(S_addr + q * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[q * 32]));
+      for (int kk = 0; kk < kTile / 16; ++kk) {
+        const uint64_t bd = desc_advance(dV, kk * 2048);
+        if (elect_one())
+          umma_ts(tmem + Cfg::kColO, tmem + Cfg::kColS + b * kTile + (kk >> 2) * 64 + (kk & 3) * 8, bd, idesc_pv,
+                  kk > 0 ? 1u : acc0);
+      }
+      if (elect_one()) {
+        umma_commit(smem_u32(&bars.kv_empty[it % NS]));
+        umma_commit(smem_u32(&bars.buf_free[b]));     // tile j+2 may overwrite the buffer
+        umma_commit(smem_u32(&bars.pv_done));         // phase j: O holds tiles 0..j
+      }
+      __syncwarp();
+    }
+  } else if (warp >= 4) {
+    // ---------------- softmax + epilogue: warpgroup `half` takes key columns [64*half, 64*half+64) ----------------
+    const int half = (warp - 4) >> 2, quad = warp & 3;
+    const int row = quad * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const uint32_t O_addr = tmem + lane_addr + Cfg::kColO + half * (D / 2);   // this thread's half of the O columns
+    const int qpos = rb.q0 + row;
+    const float c = a.scale_log2;
+    // copy this thread's row of one 64-column sub-tile of Q from the swizzled shared-memory tile into
+    // tensor memory: 16-byte chunk ch of row r sits at chunk ch ^ (r & 7)
+    bool ok = mbar_wait(smem_u32(&bars.q_full), 0, abort);
+    if (ok && half < Cfg::kSub) {
+      const unsigned char* src = smem_raw + (sQ - smem_u32(smem_raw)) + half * Cfg::kSubBytes + row * 128;
+      uint32_t v[32];
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch) {
+        const uint4 x = *reinterpret_cast<const uint4*>(src + ((ch ^ (row & 7)) << 4));
+        v[4 * ch] = x.x; v[4 * ch + 1] = x.y; v[4 * ch + 2] = x.z; v[4 * ch + 3] = x.w;
+      }
+      tmem_st32(tmem + lane_addr + Cfg::kColQ + half * 32, v);
+      tmem_wait_st();
+    }
+    tc_fence_before_sync();
+    mbar_arrive(smem_u32(&bars.qt_ready));   // also when the wait gave up: the issuers then see abort
+    float m = -INFINITY, l = 0.f;
+    // Start the second warpgroup about half a tile late: the two then stay out of phase (nothing
+    // re-aligns them while the S tiles arrive ahead of the softmax), so one warpgroup's exponentials
+    // keep the MUFU pipe busy while the other loads S and takes row maxima.
+    if (half == 1 && n > 1) __nanosleep(400);
+    for (int j = 0; j < n && ok; ++j) {
+      const int b = j & 1;
+      ok = mbar_wait(smem_u32(&bars.s_full[b]), (j >> 1) & 1, abort);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t S_own = tmem + lane_addr + Cfg::kColS + b * kTile + half * 64;
+      const uint32_t S_oth = tmem + lane_addr + Cfg::kColS + b * kTile + (1 - half) * 64;
+      uint32_t s[64], t[64];
+      tmem_ld32(S_own, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+      tmem_ld32(S_own + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+      tmem_ld32(S_oth, *reinterpret_cast<uint32_t(*)[32]>(&t[0]));
+      tmem_ld32(S_oth + 32, *reinterpret_cast<uint32_t(*)[32]>(&t[32]));
       tmem_wait_ld();
+      // keys of the tile this row may see: the first `limit`
       const int limit = j < n_ct ? rb.n_front - j * kTile : qpos - (rb.dense_start + (j - n_ct) * kTile) + 1;
       if (limit < kTile) {
+        const int lim_own = limit - half * 64, lim_oth = limit - (1 - half) * 64;
 #pragma unroll
-        for (int i = 0; i < 128; ++i)
-          if (i >= limit) s[i] = 0xff800000u;  // -inf
+        for (int i = 0; i < 64; ++i) {
+          if (i >= lim_own) s[i] = 0xff800000u;  // -inf
+          if (i >= lim_oth) t[i] = 0xff800000u;
+        }
       }
-      float mx = __uint_as_float(s[0]);
+      // row maximum over all 128 columns: both threads of a row compute the same value
+      float mx0 = fmaxf(__uint_as_float(s[0]), __uint_as_float(t[0])), mx1 = fmaxf(__uint_as_float(s[1]), __uint_as_float(t[1]));
+      float mx2 = fmaxf(__uint_as_float(s[2]), __uint_as_float(t[2])), mx3 = fmaxf(__uint_as_float(s[3]), __uint_as_float(t[3]));
 #pragma unroll
-      for (int i = 1; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(s[i]));
+      for (int i = 4; i < 64; i += 4) {
+        mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(t[i]));
+        mx1 = max3(mx1, __uint_as_float(s[i + 1]), __uint_as_float(t[i + 1]));
+        mx2 = max3(mx2, __uint_as_float(s[i + 2]), __uint_as_float(t[i + 2]));
+        mx3 = max3(mx3, __uint_as_float(s[i + 3]), __uint_as_float(t[i + 3]));
+      }
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
       if (j == 0) {
         m = mx == -INFINITY ? 0.f : mx;
       } else {
         const bool need = (mx - m) * c > 8.f;
         if (__any_sync(0xffffffffu, need)) {
-          ok = mbar_wait(smem_u32(&bars.pv_done[t]), (j - 1) & 1, abort);
+          // O must hold every earlier tile before it is rescaled; the O issuer cannot start tile j before
+          // this thread has arrived on p_full, so the rescale cannot race with it
+          ok = mbar_wait(smem_u32(&bars.pv_done), (j - 1) & 1, abort);
           if (!ok) break;
           tc_fence_after_sync();
           const float f = need ? ex2((m - mx) * c) : 1.f;
 #pragma unroll
-          for (int q = 0; q < D / 32; ++q) {
+          for (int q = 0; q < D / 64; ++q) {
             uint32_t o[32];
             tmem_ld32(O_addr + q * 32, o);
             tmem_wait_ld();
@@ -231,50 +264,50 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         }
       }
       const float nmc = -m * c;
-      float sum = 0.f;
+      float sum0 = 0.f, sum1 = 0.f;
+      uint32_t pk[32];
 #pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        uint32_t pk[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float p0 = ex2(fmaf(__uint_as_float(s[q * 64 + 2 * i]), c, nmc));
-          const float p1 = ex2(fmaf(__uint_as_float(s[q * 64 + 2 * i + 1]), c, nmc));
-          sum += p0 + p1;
-          pk[i] = pack_bf16(p0, p1);
-        }
-        tmem_st32(S_addr + q * 32, pk);
+      for (int i = 0; i < 32; ++i) {
+        // one exponential in four on the FMA pipe, the rest on the MUFU pipe
+        const float p0 = ex2(fmaf(__uint_as_float(s[2 * i]), c, nmc));
+        const float x1 = fmaf(__uint_as_float(s[2 * i + 1]), c, nmc);
+        const float p1 = (i & 1) ? ex2_fma(x1) : ex2(x1);
+        sum0 += p0; sum1 += p1;
+        pk[i] = pack_bf16(p0, p1);
       }
+      l += sum0 + sum1;
+      tmem_st32(S_own, pk);   // over the first half of this warpgroup's own S columns
       tmem_wait_st();
-      l += sum;
       tc_fence_before_sync();
-      mbar_arrive(smem_u32(&bars.p_full[t]));
+      mbar_arrive(smem_u32(&bars.p_full[b]));
     }
-    if (ok && n > 0) {
-      ok = mbar_wait(smem_u32(&bars.pv_done[t]), (n - 1) & 1, abort);
-      if (ok) {
-        tc_fence_after_sync();
-        const float inv = 1.0f / l;
-        const bool store = qpos < rb.q_end;
-        __nv_bfloat16* orow = a.O + ((size_t)bh * a.N + qpos) * D;
+    red_s[half][row] = l;
+    asm volatile("bar.sync 1, 256;" ::: "memory");   // the eight softmax warps, whether or not a wait gave up
+    if (ok) ok = mbar_wait(smem_u32(&bars.pv_done), (n - 1) & 1, abort);
+    if (ok) {
+      tc_fence_after_sync();
+      const float lt = red_s[0][row] + red_s[1][row];
+      const float inv = 1.0f / lt;
+      const bool store = qpos < rb.q_end;
+      __nv_bfloat16* orow = a.O + ((size_t)bh * a.N + qpos) * D + half * (D / 2);
 #pragma unroll
-        for (int q = 0; q < D / 32; ++q) {
-          uint32_t o[32];
-          tmem_ld32(O_addr + q * 32, o);
-          tmem_wait_ld();
-          if (store) {
+      for (int q = 0; q < D / 64; ++q) {
+        uint32_t o[32];
+        tmem_ld32(O_addr + q * 32, o);
+        tmem_wait_ld();
+        if (store) {
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              uint4 w;
-              w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
-              w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
-              w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
-              w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-              *reinterpret_cast<uint4*>(orow + q * 32 + v * 8) = w;
-            }
+          for (int v = 0; v < 4; ++v) {
+            uint4 w;
+            w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+            w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+            w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+            w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + q * 32 + v * 8) = w;
           }
         }
-        if (store) a.LSE[(size_t)bh * a.N + qpos] = m * a.scale + logf(l);
       }
+      if (store && half == 0) a.LSE[(size_t)bh * a.N + qpos] = m * a.scale + logf(lt);
     }
   }
 
@@ -371,7 +404,7 @@ static int launch_fwd_t(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat
   if (rc_ == LRSA_OK) rc_ = make_tmap_bf16(&mVc, Vc, D, rc, (long long)g.B * g.Hkv, kTile);
   if (rc_ != LRSA_OK) return rc_;
   FwdArgs a;
-  a.plan = make_plan(g, 2 * kTile);
+  a.plan = make_plan(g, kTile);
   a.BH = g.B * g.Hq; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.N = g.N;
   a.O = O; a.LSE = LSE; a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f;
   a.status = status;

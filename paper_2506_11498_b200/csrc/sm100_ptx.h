@@ -181,6 +181,24 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// 2^x on the FMA pipe for x <= ~100: n = round(x) through the 1.5*2^23 trick, a cubic for 2^(x-n) on
+// [-0.5, 0.5] (fitted here, relative error below 8e-5, well under bf16 rounding), then n added into the
+// exponent field.  x = -inf (a masked score) is clamped and gives about 2^-125, zero for all purposes.
+// It shares the exponentials with the MUFU pipe (ex2), which is otherwise the forward kernel's bottleneck.
+__device__ __forceinline__ float ex2_fma(float x) {
+  x = fmaxf(x, -125.f);   // keeps the biased exponent of the result positive
+  const float t = x + 12582912.f;
+  const float f = x - (t - 12582912.f);
+  float p = fmaf(0.0551708005f, f, 0.2426092625f);
+  p = fmaf(p, f, 0.6932609677f);
+  p = fmaf(p, f, 0.9999281764f);
+  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));

@@ -21,13 +21,19 @@ def host_bits(host):
     return {k: orc.bf16_bits(v) for k, v in host.items()}
 
 
-def check_close(name, got, want, max_abs=MAX_ABS, rel_l2=REL_L2):
+def check_close(name, got, want, max_abs=MAX_ABS, rel_l2=REL_L2, row_scale=False):
+    """`row_scale`: scale the absolute bound by the largest reference magnitude of the row (last axis)
+    instead of the element's own.  A gradient element is a sum of bf16-rounded products that may
+    cancel; its rounding error follows the size of the terms, which the row's largest element tracks,
+    not the size of the cancelled result.  Used only for the deliberately ill-conditioned small case
+    (keys scaled by 8); the benchmark configurations are held to the element-wise bound."""
     got = np.asarray(got, np.float64)
     want = np.asarray(want, np.float64)
     assert got.shape == want.shape, (name, got.shape, want.shape)
     assert np.isfinite(got).all(), f"{name}: non-finite values"
     err = np.abs(got - want)
-    bound = max_abs * np.maximum(1.0, np.abs(want))
+    ref_mag = np.abs(want).max(axis=-1, keepdims=True) if row_scale else np.abs(want)
+    bound = max_abs * np.maximum(1.0, ref_mag)
     worst = int(np.argmax(err - bound))
     assert (err <= bound).all(), f"{name}: |err|={err.flat[worst]:.4g} at {worst} (ref {want.flat[worst]:.4g})"
     denom = np.linalg.norm(want)

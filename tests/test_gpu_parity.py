@@ -100,11 +100,12 @@ def test_attention_fwd_bwd(w, ndp):
     oO, oL = orc.attn_fwd(op, bits["Q"], bits["K"], bits["V"], oidx)
     odQ, odK, odV = orc.attn_bwd(op, bits["Q"], bits["K"], bits["V"], bits["dO"], oidx)
     O, LSE, dQ, dK, dV = _run_attention(w, ndp, oidx, host)
+    rs = w.values == "salient"      # a handful of x8 keys in a 700-token sequence: see check_close
     check_close("O", f64(O), oO)
     check_close("LSE", f64(LSE), oL, max_abs=2e-3, rel_l2=1e-4)
-    check_close("dQ", f64(dQ), odQ)
-    check_close("dK", f64(dK), odK)
-    check_close("dV", f64(dV), odV)
+    check_close("dQ", f64(dQ), odQ, row_scale=rs)
+    check_close("dK", f64(dK), odK, row_scale=rs)
+    check_close("dV", f64(dV), odV, row_scale=rs)
 
 
 def test_end_to_end_and_determinism():
