@@ -16,6 +16,7 @@
 // therefore picked up by CTAs that already run, and publish before they wait on anything: the
 // wait always ends, whatever the number of resident CTAs.  It is bounded all the same.
 #include "lrsa_internal.h"
+#include "sm100_ptx.h"
 
 namespace lrsa {
 namespace {
@@ -75,30 +76,38 @@ __device__ __forceinline__ float warp_sum(float v) {
 }
 
 // Top-K of the window by the last CTA to finish it.  smem: sk[L], sv[L] floats, then scratch.
-__device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* smem) {
+// Bytes of the selection scratch: sk[L], sv[L], 256 histogram bins, 32 floats, 16 ints.
+__host__ __device__ inline size_t select_scratch_bytes(int L) { return (size_t)2 * L * 4 + 256 * 4 + 32 * 4 + 16 * 4; }
+
+// Barrier of the 256 scoring threads (named barrier 1): the whole block in the one-unit-per-CTA kernel,
+// all warps but the producer in the streaming kernel.
+__device__ __forceinline__ void scoring_warps_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// `in_smem`: the spreads are already in sk / sv (the chain kernel keeps them there) instead of in a.spread.
+__device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* smem, bool in_smem = false) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, L = a.L;
   float* sk = reinterpret_cast<float*>(smem);
   float* sv = sk + L;
   uint32_t* hist = reinterpret_cast<uint32_t*>(sv + L);  // 256 bins
   float* red = reinterpret_cast<float*>(hist + 256);     // 32 floats
   int* ibuf = reinterpret_cast<int*>(red + 32);          // 16 ints
-  const float* gk = a.spread + ((size_t)(bh * a.Wsel + w) * 2 + 0) * L;
-  const float* gv = gk + L;
+  const float* gk = in_smem ? sk : a.spread + ((size_t)(bh * a.Wsel + w) * 2 + 0) * L;
+  const float* gv = in_smem ? sv : gk + L;
 
   // Eq. 7: softmax over the L tokens of the window, for K and for V
   float mk = -INFINITY, mv = -INFINITY;
   for (int i = tid; i < L; i += kThreads) {
-    const float x = __ldcg(gk + i), y = __ldcg(gv + i);
+    const float x = in_smem ? sk[i] : __ldcg(gk + i), y = in_smem ? sv[i] : __ldcg(gv + i);
     sk[i] = x; sv[i] = y;
     mk = fmaxf(mk, x); mv = fmaxf(mv, y);
   }
   mk = warp_max(mk); mv = warp_max(mv);
   if (lane == 0) { red[warp] = mk; red[8 + warp] = mv; }
-  __syncthreads();
+  scoring_warps_sync();
   mk = red[0]; mv = red[8];
 #pragma unroll
   for (int i = 1; i < 8; ++i) { mk = fmaxf(mk, red[i]); mv = fmaxf(mv, red[8 + i]); }
-  __syncthreads();
+  scoring_warps_sync();
   float ek = 0.f, ev = 0.f;
   for (int i = tid; i < L; i += kThreads) {
     const float x = expf(sk[i] - mk), y = expf(sv[i] - mv);
@@ -107,7 +116,7 @@ __device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* 
   }
   ek = warp_sum(ek); ev = warp_sum(ev);
   if (lane == 0) { red[warp] = ek; red[8 + warp] = ev; }
-  __syncthreads();
+  scoring_warps_sync();
   ek = 0.f; ev = 0.f;
 #pragma unroll
   for (int i = 0; i < 8; ++i) { ek += red[i]; ev += red[8 + i]; }
@@ -118,7 +127,7 @@ __device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* 
     sk[i] = s;
     if (gs) gs[i] = s;
   }
-  __syncthreads();
+  scoring_warps_sync();
 
   // radix select of the K-th largest score; scores are positive, so bit order = value order
   const uint32_t* key = reinterpret_cast<const uint32_t*>(sk);
@@ -126,12 +135,12 @@ __device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* 
   int remaining = a.Kk;
   for (int shift = 24; shift >= 0; shift -= 8) {
     hist[tid] = 0;
-    __syncthreads();
+    scoring_warps_sync();
     for (int i = tid; i < L; i += kThreads) {
       const uint32_t k = key[i];
       if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1u);
     }
-    __syncthreads();
+    scoring_warps_sync();
     if (warp == 0) {
       // lane l owns bins 255-8l ... 248-8l, highest first
       uint32_t c[8], tot = 0;
@@ -151,11 +160,11 @@ __device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* 
         ibuf[1] = remaining - (int)above;
       }
     }
-    __syncthreads();
+    scoring_warps_sync();
     prefix |= (uint32_t)ibuf[0] << shift;
     mask |= 255u << shift;
     remaining = ibuf[1];
-    __syncthreads();
+    scoring_warps_sync();
   }
   const uint32_t kth = prefix;    // K-th largest key
   const int need_eq = remaining;  // how many keys equal to it are kept (lowest positions first)
@@ -176,7 +185,7 @@ __device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* 
       if (lane >= o) incl += n;
     }
     if (lane == 31) wtot[warp] = incl;
-    __syncthreads();
+    scoring_warps_sync();
     int excl = incl - packed, all = 0;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
@@ -189,7 +198,7 @@ __device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* 
       out[gt_before + min(eq_before, need_eq)] = a.S + w * L + i;
     base_gt += all & 0xffff;
     base_eq += all >> 16;
-    __syncthreads();
+    scoring_warps_sync();
   }
 }
 
@@ -351,6 +360,240 @@ __global__ void __launch_bounds__(kThreads) score_select_kernel(const ScoreArgs 
   select_window(a, bh, w, smem);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Chain kernel (lag windows up to kChainMaxL tokens): no communication between CTAs at all.
+//
+// A CTA owns a run of consecutive scored windows [w_a, w_b) of one (batch, KV head) and walks it
+// downwards.  It first streams window w_b only for its channel minima and maxima (Eq. 4-5); then for
+// w = w_b-1 ... w_a every 16 KB slice of K and of V is normalised with the statistics of window w+1,
+// already in shared memory (Eq. 6), reduced to per-token spreads (Eq. 7) that stay in shared memory,
+// and folded into the running statistics of window w itself for the next step; at the end of a
+// window the CTA soft-maxes, adds (Eq. 8) and selects.  A producer warp keeps a ring of slices in
+// flight with bulk asynchronous copies, so the loads never wait for the arithmetic; two groups of
+// eight scoring warps take alternate slices (the arithmetic of one slice is a chain of dependent
+// shuffles and reductions, and one group alone leaves the SM idle most of the time).
+// With one window per CTA (the 32K benchmark: 120 windows on 148 SMs) every window is streamed
+// twice, by its own CTA and as the reference of the window before it; the second read comes a few
+// microseconds after the first and is served by L2 as long as K and V fit there (67 MB of 126 MB).
+// Longer runs per CTA (more windows than SMs) read 1 + 1/run of the data.
+constexpr int kChainStages = 5;
+constexpr int kChainMaxL = 4096;
+constexpr int kChainGroups = 2;                           // scoring groups of kThreads threads, alternating slices
+constexpr int kChainThreads = kChainGroups * kThreads + 32;
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void group_sync(int grp) { asm volatile("bar.sync %0, 256;" ::"r"(grp + 1) : "memory"); }
+__device__ __forceinline__ void all_groups_sync() {
+  asm volatile("bar.sync 3, %0;" ::"n"(kChainGroups * kThreads) : "memory");
+}
+
+// Bounded wait on a shared-memory barrier phase; false when it gave up.
+__device__ __forceinline__ bool stage_wait(uint32_t bar, uint32_t parity, int limit) {
+  for (int it = 0; it < limit; ++it)
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(const ScoreArgs a, int run, int runs_per_bh) {
+  constexpr int LPR = D / 8;              // lanes per token row, 16 bytes each
+  constexpr int RPS = kThreads / LPR;     // rows per step
+  constexpr int TOK = kSteps * RPS;       // tokens per slice
+  constexpr int kSliceBytes = TOK * D * 2;
+  constexpr int kStageBytes = 2 * kSliceBytes;   // K slice, then V slice
+  extern __shared__ __align__(16) unsigned char smem[];
+  __shared__ __align__(8) uint64_t full_bar[kChainStages], empty_bar[kChainStages];
+  __shared__ int s_abort;
+  // after the ring: scale/offset of the reference window [2 (K,V)][2 (sa,sb)][D], then the selection
+  // scratch (spreads sk[L], sv[L], histogram...), whose tail doubles as the min/max reduction buffer
+  float* sasb = reinterpret_cast<float*>(smem + kChainStages * kStageBytes);
+  unsigned char* sel = reinterpret_cast<unsigned char*>(sasb + 4 * D);
+  float* sk = reinterpret_cast<float*>(sel);
+  float* sv = sk + a.L;
+  __nv_bfloat16* red = reinterpret_cast<__nv_bfloat16*>(sel + select_scratch_bytes(a.L));   // [16 warps][4][D]
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    s_abort = 0;
+    for (int i = 0; i < kChainStages; ++i) {
+      ptx::mbar_init(ptx::smem_u32(&full_bar[i]), 1);
+      ptx::mbar_init(ptx::smem_u32(&empty_bar[i]), 1);
+    }
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+  const int bh = blockIdx.x / runs_per_bh, seg = blockIdx.x % runs_per_bh;
+  const int w_a = seg * run, w_b = min(a.Wsel, w_a + run);   // scored windows [w_a, w_b); reference w_b <= W-1
+  const int n_win = w_b - w_a + 1;                            // windows streamed, the reference first
+  const int n_it = n_win * a.n_slices;
+  volatile int* abort = &s_abort;
+
+  if (warp == kChainGroups * kThreads / 32) {
+    // ---------------- producer ----------------
+    if (lane != 0) return;
+    for (int i = 0; i < n_it; ++i) {
+      const int slot = i % kChainStages;
+      if (i >= kChainStages &&
+          !stage_wait(ptx::smem_u32(&empty_bar[slot]), ((i / kChainStages) - 1) & 1, a.spin_limit)) {
+        *abort = 1;
+        atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT);
+        return;
+      }
+      if (*abort) return;
+      const int w = w_b - i / a.n_slices, slice = i % a.n_slices;
+      const int rows = min(TOK, a.L - slice * TOK);
+      const uint32_t bytes = (uint32_t)rows * D * 2;
+      const size_t off = ((size_t)bh * a.N + a.S + (size_t)w * a.L + (size_t)slice * TOK) * D;
+      const uint32_t bar = ptx::smem_u32(&full_bar[slot]);
+      const uint32_t dst = ptx::smem_u32(smem + slot * kStageBytes);
+      ptx::mbar_expect_tx(bar, 2 * bytes);
+      bulk_load(dst, a.K + off, bytes, bar);
+      bulk_load(dst + kSliceBytes, a.V + off, bytes, bar);
+    }
+    return;
+  }
+
+  // ---------------- scoring warps ----------------
+  const int grp = tid / kThreads, gt = tid % kThreads;   // group and thread within the group
+  const int chunk = gt % LPR, row = gt / LPR;
+  const float inv_dof = 1.0f / (float)(D - a.ddof);
+  const uint32_t PINF = 0x7F807F80u, NINF = 0xFF80FF80u;
+  uint32_t st[2][2][4];  // running [K,V][min,max][4 bf16 pairs] of this group's slices of the window
+  for (int wi = 0; wi < n_win; ++wi) {
+   const int w = w_b - wi;
+   const bool scoring = wi > 0;          // the first window streamed is a reference only
+   const bool want_stats = w > w_a;      // its statistics serve the next window of the run
+#pragma unroll
+   for (int j = 0; j < 4; ++j) { st[0][0][j] = st[1][0][j] = PINF; st[0][1][j] = st[1][1][j] = NINF; }
+   for (int i = wi * a.n_slices; i < (wi + 1) * a.n_slices; ++i) {
+    if (i % kChainGroups != grp) continue;
+    const int slice = i % a.n_slices;
+    const int slot = i % kChainStages;
+    if (!stage_wait(ptx::smem_u32(&full_bar[slot]), (i / kChainStages) & 1, a.spin_limit)) {
+      *abort = 1;
+      atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT);
+    }
+    group_sync(grp);
+    if (*abort) break;   // the same verdict for every thread of the group: it was written before the barrier
+    const unsigned char* stage = smem + slot * kStageBytes;
+    // this thread's rows of the slice: kSteps rows of K and of V, 16 bytes (8 channels) each
+    uint4 kq[kSteps], vq[kSteps];
+    bool valid[kSteps];
+#pragma unroll
+    for (int s = 0; s < kSteps; ++s) {
+      const int t = s * RPS + row;
+      valid[s] = slice * TOK + t < a.L;
+      if (valid[s]) {
+        kq[s] = *reinterpret_cast<const uint4*>(stage + (size_t)t * D * 2 + chunk * 16);
+        vq[s] = *reinterpret_cast<const uint4*>(stage + kSliceBytes + (size_t)t * D * 2 + chunk * 16);
+      } else {
+        kq[s] = make_uint4(0, 0, 0, 0);
+        vq[s] = make_uint4(0, 0, 0, 0);
+      }
+    }
+    if (want_stats) {
+      // Eq. 4, Eq. 5, folded into the running statistics
+#pragma unroll
+      for (int s = 0; s < kSteps; ++s) {
+        if (!valid[s]) continue;
+        const uint32_t kk[4] = {kq[s].x, kq[s].y, kq[s].z, kq[s].w}, vv[4] = {vq[s].x, vq[s].y, vq[s].z, vq[s].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          st[0][0][j] = bmin2(st[0][0][j], kk[j]); st[0][1][j] = bmax2(st[0][1][j], kk[j]);
+          st[1][0][j] = bmin2(st[1][0][j], vv[j]); st[1][1][j] = bmax2(st[1][1][j], vv[j]);
+        }
+      }
+    }
+    if (scoring) {
+      // Eq. 6 with the statistics of window w+1 (z' = x*sa + sb = zbar - 1/2) and the per-token Std of Eq. 7
+#pragma unroll
+      for (int z = 0; z < 2; ++z) {
+        float sa[8], sb[8];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float4 va = *reinterpret_cast<const float4*>(sasb + (z * 2 + 0) * D + chunk * 8 + h * 4);
+          const float4 vb = *reinterpret_cast<const float4*>(sasb + (z * 2 + 1) * D + chunk * 8 + h * 4);
+          sa[h * 4 + 0] = va.x; sa[h * 4 + 1] = va.y; sa[h * 4 + 2] = va.z; sa[h * 4 + 3] = va.w;
+          sb[h * 4 + 0] = vb.x; sb[h * 4 + 1] = vb.y; sb[h * 4 + 2] = vb.z; sb[h * 4 + 3] = vb.w;
+        }
+        float* out = z == 0 ? sk : sv;
+#pragma unroll
+        for (int s = 0; s < kSteps; ++s) {
+          const uint4 q = z == 0 ? kq[s] : vq[s];
+          const uint32_t pk[4] = {q.x, q.y, q.z, q.w};
+          float sum = 0.f, sq = 0.f;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float z0 = fmaf(bf_lo(pk[j]), sa[2 * j], sb[2 * j]);
+            const float z1 = fmaf(bf_hi(pk[j]), sa[2 * j + 1], sb[2 * j + 1]);
+            sum += z0 + z1;
+            sq = fmaf(z0, z0, sq);
+            sq = fmaf(z1, z1, sq);
+          }
+#pragma unroll
+          for (int o = LPR / 2; o > 0; o >>= 1) {
+            sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            sq += __shfl_xor_sync(0xffffffffu, sq, o);
+          }
+          if (chunk == 0 && valid[s]) {
+            const float var = (sq - sum * sum * (1.0f / D)) * inv_dof;
+            out[slice * TOK + s * RPS + row] = sqrtf(fmaxf(var, 0.f));
+          }
+        }
+      }
+    }
+    group_sync(grp);   // every read of the stage by this group is done
+    if (gt == 0) ptx::mbar_arrive(ptx::smem_u32(&empty_bar[slot]));
+   }
+
+   // ---- end of window w: both groups have written their spreads and hold their part of the statistics ----
+   all_groups_sync();
+   if (*abort) return;   // set before the barrier by whichever thread gave up
+   if (scoring && grp == 0) select_window(a, bh, w, sel, true);   // group 0 only (its own barrier inside)
+   if (want_stats) {
+      // reduce the running statistics over the rows of a warp, then over the warps, and turn them
+      // into the scale and offset the next window is normalised with
+#pragma unroll
+      for (int o = 16; o >= LPR; o >>= 1)
+#pragma unroll
+        for (int z = 0; z < 2; ++z)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            st[z][0][j] = bmin2(st[z][0][j], __shfl_xor_sync(0xffffffffu, st[z][0][j], o));
+            st[z][1][j] = bmax2(st[z][1][j], __shfl_xor_sync(0xffffffffu, st[z][1][j], o));
+          }
+      if (lane < LPR) {
+#pragma unroll
+        for (int z = 0; z < 2; ++z)
+#pragma unroll
+          for (int m = 0; m < 2; ++m)
+            *reinterpret_cast<uint4*>(red + ((warp * 4 + z * 2 + m) * D + lane * 8)) =
+                make_uint4(st[z][m][0], st[z][m][1], st[z][m][2], st[z][m][3]);
+      }
+      all_groups_sync();
+      for (int v = tid; v < 2 * D; v += kChainGroups * kThreads) {
+        const int z = v / D, ch = v % D;
+        float mn = __bfloat162float(red[(z * 2 + 0) * D + ch]), mx = __bfloat162float(red[(z * 2 + 1) * D + ch]);
+#pragma unroll
+        for (int ww = 1; ww < kChainGroups * kThreads / 32; ++ww) {
+          mn = fminf(mn, __bfloat162float(red[(ww * 4 + z * 2 + 0) * D + ch]));
+          mx = fmaxf(mx, __bfloat162float(red[(ww * 4 + z * 2 + 1) * D + ch]));
+        }
+        // a channel with zero range has zbar = 0, i.e. z' = -1/2
+        const float range = mx - mn;
+        const float inv = range > 0.f ? 1.0f / range : 0.f;
+        sasb[(z * 2 + 0) * D + ch] = inv;
+        sasb[(z * 2 + 1) * D + ch] = range > 0.f ? -(0.5f * (mn + mx)) * inv : -0.5f;
+      }
+   }
+   all_groups_sync();   // the next window's slices may overwrite the spreads and read the new statistics
+  }
+}
+
 template <int D>
 constexpr int tok_per_unit() { return kSteps * (kThreads / (D / 8)); }
 
@@ -385,7 +628,8 @@ int launch_score_select(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat
   if (g.Wsel == 0) return LRSA_OK;  // nothing is scored
   const ScoreWs lay = score_ws_layout(g);
   unsigned char* base = static_cast<unsigned char*>(ws);
-  LRSA_CUDA_CHECK(cudaMemsetAsync(base, 0, lay.zero_bytes, st));
+  // the chain kernel keeps everything but the status word on chip
+  LRSA_CUDA_CHECK(cudaMemsetAsync(base, 0, g.L <= kChainMaxL ? sizeof(WsHeader) : lay.zero_bytes, st));
   launch_counter().n++;
   ScoreArgs a;
   a.K = K; a.V = V; a.idx = idx; a.score = score;
@@ -403,6 +647,24 @@ int launch_score_select(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat
   if (smem > 200 * 1024) return LRSA_ERR_UNSUPPORTED;
   const long long units = (long long)a.BH * g.W * a.n_slices;
   if (units > 0x7fffffffLL) return LRSA_ERR_UNSUPPORTED;
+  if (g.L <= kChainMaxL) {
+    // chain kernel: runs of consecutive windows per CTA, about one CTA per SM, no inter-CTA traffic
+    int dev = 0, sms = 0;
+    LRSA_CUDA_CHECK(cudaGetDevice(&dev));
+    LRSA_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int run = (a.BH * g.Wsel + sms - 1) / sms;
+    const int runs_per_bh = (g.Wsel + run - 1) / run;
+    const size_t bytes = (size_t)kChainStages * 2 * tok * g.d * sizeof(__nv_bfloat16)   // ring
+                         + (size_t)4 * g.d * sizeof(float)                               // scale / offset
+                         + select_scratch_bytes(g.L)
+                         + (size_t)(kChainGroups * kThreads / 32) * 4 * g.d * sizeof(__nv_bfloat16);   // min/max reduction
+    auto ckern = g.d == 128 ? score_select_chain_kernel<128> : score_select_chain_kernel<64>;
+    LRSA_CUDA_CHECK(cudaFuncSetAttribute(ckern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    ckern<<<(unsigned)(a.BH * runs_per_bh), kChainThreads, bytes, st>>>(a, run, runs_per_bh);
+    LRSA_CUDA_CHECK(cudaGetLastError());
+    launch_counter().n++;
+    return LRSA_OK;
+  }
   auto kern = g.d == 128 ? score_select_kernel<128> : score_select_kernel<64>;
   LRSA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   kern<<<(unsigned)units, kThreads, smem, st>>>(a);
