@@ -23,6 +23,9 @@ SCORE_CASES = [
     W("s_offsets", 1, 4, 2, 4 + 8 * 1024, 128, 1024, 256, 4, seed=17, values="channel_offset"),
     W("s_salient", 1, 2, 2, 4 + 4 * 2048 + 9, 128, 2048, 512, 4, seed=18, values="salient"),
     W("s_tiny_window", 1, 1, 1, 70, 64, 8, 3, 1, seed=19),
+    # lag windows beyond 4096 tokens take the one-slice-per-CTA kernel with global statistics
+    W("s_long_window", 1, 1, 1, 2 + 3 * 4608 + 11, 64, 4608, 100, 2, seed=42),
+    W("s_long_window128", 1, 2, 1, 4 * 4160, 128, 4160, 4000, 0, seed=43),
 ]
 
 
