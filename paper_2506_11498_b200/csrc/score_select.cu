@@ -450,6 +450,14 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
       const size_t off = ((size_t)bh * a.N + a.S + (size_t)w * a.L + (size_t)slice * TOK) * D;
       const uint32_t bar = ptx::smem_u32(&full_bar[slot]);
       const uint32_t dst = ptx::smem_u32(smem + slot * kStageBytes);
+      // self-check: the slice lies inside the tensor and the copy is 16-byte granular; otherwise give up
+      // (status word) instead of issuing it
+      if (w < 0 || w >= a.W || rows <= 0 || off + (size_t)rows * D > (size_t)a.BH * a.N * D || (bytes & 15u) ||
+          ((reinterpret_cast<uintptr_t>(a.K + off) | reinterpret_cast<uintptr_t>(a.V + off) | dst) & 15u)) {
+        *abort = 1;
+        atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT);
+        return;
+      }
       ptx::mbar_expect_tx(bar, 2 * bytes);
       bulk_load(dst, a.K + off, bytes, bar);
       bulk_load(dst + kSliceBytes, a.V + off, bytes, bar);
