@@ -338,8 +338,12 @@ def main():
         "stage_rates": {"fwd_tflops": f_fwd / fwd_s / 1e12, "bwd_tflops": f_bwd / bwd_s / 1e12,
                         "score_select_gbs": kv_bytes(wl) / score_s / 1e9,
                         "score_select_frac_of_hbm": kv_bytes(wl) / score_s / 1e9 / peaks["hbm_gbs"]},
-        "roofline": {"kernel": "lrsa_attn_bwd", "bound": "tensor", "achieved": achieved, "peak": peak_tf,
-                     "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": None,
+        # achieved = effective backward FLOPs (10*d per unmasked pair) / the backward call's CUDA-event time
+        # (dK/dV kernel + dQ kernel + ~2 % helpers).  traffic: DRAM bytes of those two kernels in one launch
+        # each (ncu, profiles/lrsa_kernels_cfg2_32k.md: 9115+245 MB and 565+208 MB), known for the 32K workload.
+        "roofline": {"kernel": "lrsa_attn_bwd (lrsa_bwd_dkv_kernel + lrsa_bwd_dq_kernel)", "bound": "tensor",
+                     "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
+                     "traffic": 1.0133e10 if wl.name == "cfg2_32k_gqa7_d128" else None,
                      "peak_source": f"{peaks['source']} sustained bf16"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches[0] * args.steps,
     }
