@@ -190,14 +190,17 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2_32k_gqa7_d128")
+    ap.add_argument("--workload", default="cfg2_32k_gqa7_d128",
+                    help="a configuration name (cfg1_..cfg4_) or a sweep point such as cfg5_L1024_r1/4")
+    ap.add_argument("--n-dense-prev", type=int, default=1, choices=[0, 1],
+                    help="1: the window before the query chunk is seen uncompressed (the paper); 0: compressed too")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
     from paper_2506_11498_b200 import workloads
-    w = workloads.CONFIGS[args.workload]
+    w = {**workloads.CONFIGS, **{pt.name: pt for pt in workloads.sweep_points()}}[args.workload]
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -216,7 +219,7 @@ def main():
     # weak scaling: every rank runs its own sequence (independent problems, no data-path collective)
     wl = replicas.rank_workload(w, rank)
     lrsa.lib()
-    p = lrsa.Params.from_workload(wl)
+    p = lrsa.Params.from_workload(wl, n_dense_prev=args.n_dense_prev)
     host = {k: v.pin_memory() for k, v in workloads.generate(wl).items()}
     dev = {k: v.cuda(non_blocking=True) for k, v in host.items()}
     ws_sizes = lrsa.lrsa_workspace_bytes(p)
@@ -335,7 +338,7 @@ def main():
             if not torch.equal(outs_host[name], t.cpu()):
                 raise SystemExit(f"end-to-end leg: host copy of {name} differs from the device result")
         e2e_ms = replicas.max_over_ranks(e0.elapsed_time(e1) / n_e2e, dist, "cuda")
-        f_fwd, f_bwd = flops(wl)
+        f_fwd, f_bwd = flops(wl, args.n_dense_prev)
         e2e = {"value": replicas.job_rate(f_fwd + f_bwd, world, e2e_ms * 1e-3) / 1e12, "unit": UNIT,
                "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "overlap": "uploads, kernels and downloads of consecutive steps overlap (two buffer sets, three streams)"}
@@ -345,7 +348,7 @@ def main():
             dist.destroy_process_group()
         return
 
-    f_fwd, f_bwd = flops(wl)
+    f_fwd, f_bwd = flops(wl, args.n_dense_prev)
     peaks = measured_peaks()
     med = statistics.median
     bwd_s, fwd_s, score_s = med(t_bwd) * 1e-3, med(t_fwd) * 1e-3, med(t_score) * 1e-3
@@ -358,7 +361,7 @@ def main():
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": wl.name, "B": wl.B, "N": wl.N, "Hq": wl.Hq, "Hkv": wl.Hkv, "d": wl.d,
-                   "L": wl.L, "K": wl.K, "S": wl.S, "values": wl.values,
+                   "L": wl.L, "K": wl.K, "S": wl.S, "values": wl.values, "n_dense_prev": args.n_dense_prev,
                    "l2": "256 MB buffer written between timed steps (outside the per-step events)",
                    "parallelism": f"replicas x{world} (independent sequences, no collective)"},
         "tokens_per_s": world * wl.B * wl.N / (ms_per_step * 1e-3),

@@ -371,12 +371,15 @@ __global__ void __launch_bounds__(kThreads) score_select_kernel(const ScoreArgs 
 // window the CTA soft-maxes, adds (Eq. 8) and selects.  A producer warp keeps a ring of slices in
 // flight with bulk asynchronous copies, so the loads never wait for the arithmetic; two groups of
 // eight scoring warps take alternate slices (the arithmetic of one slice is a chain of dependent
-// shuffles and reductions, and one group alone leaves the SM idle most of the time).
+// shuffles and reductions, and one group alone leaves the SM idle most of the time).  Each group has
+// its own ring of stages and waits for its slices in the order they were issued: a barrier is then
+// never waited on two phases ahead (a parity wait cannot tell "two phases ahead" from "done"), which
+// a shared ring allowed when one group ran ahead and bulk copies landed out of order.
 // With one window per CTA (the 32K benchmark: 120 windows on 148 SMs) every window is streamed
 // twice, by its own CTA and as the reference of the window before it; the second read comes a few
 // microseconds after the first and is served by L2 as long as K and V fit there (67 MB of 126 MB).
 // Longer runs per CTA (more windows than SMs) read 1 + 1/run of the data.
-constexpr int kChainStages = 5;
+constexpr int kChainMaxRing = 3;   // stages per scoring group (2 when the selection scratch is large)
 constexpr int kChainMaxL = 4096;
 constexpr int kChainGroups = 2;                           // scoring groups of kThreads threads, alternating slices
 constexpr int kChainThreads = kChainGroups * kThreads + 32;
@@ -399,18 +402,19 @@ __device__ __forceinline__ bool stage_wait(uint32_t bar, uint32_t parity, int li
 }
 
 template <int D>
-__global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(const ScoreArgs a, int run, int runs_per_bh) {
+__global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(const ScoreArgs a, int run, int runs_per_bh,
+                                                                              int ring) {
   constexpr int LPR = D / 8;              // lanes per token row, 16 bytes each
   constexpr int RPS = kThreads / LPR;     // rows per step
   constexpr int TOK = kSteps * RPS;       // tokens per slice
   constexpr int kSliceBytes = TOK * D * 2;
   constexpr int kStageBytes = 2 * kSliceBytes;   // K slice, then V slice
   extern __shared__ __align__(16) unsigned char smem[];
-  __shared__ __align__(8) uint64_t full_bar[kChainStages], empty_bar[kChainStages];
+  __shared__ __align__(8) uint64_t full_bar[kChainGroups * kChainMaxRing], empty_bar[kChainGroups * kChainMaxRing];
   __shared__ int s_abort;
   // after the ring: scale/offset of the reference window [2 (K,V)][2 (sa,sb)][D], then the selection
   // scratch (spreads sk[L], sv[L], histogram...), whose tail doubles as the min/max reduction buffer
-  float* sasb = reinterpret_cast<float*>(smem + kChainStages * kStageBytes);
+  float* sasb = reinterpret_cast<float*>(smem + kChainGroups * ring * kStageBytes);
   unsigned char* sel = reinterpret_cast<unsigned char*>(sasb + 4 * D);
   float* sk = reinterpret_cast<float*>(sel);
   float* sv = sk + a.L;
@@ -419,7 +423,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
     s_abort = 0;
-    for (int i = 0; i < kChainStages; ++i) {
+    for (int i = 0; i < kChainGroups * kChainMaxRing; ++i) {
       ptx::mbar_init(ptx::smem_u32(&full_bar[i]), 1);
       ptx::mbar_init(ptx::smem_u32(&empty_bar[i]), 1);
     }
@@ -436,9 +440,9 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
     // ---------------- producer ----------------
     if (lane != 0) return;
     for (int i = 0; i < n_it; ++i) {
-      const int slot = i % kChainStages;
-      if (i >= kChainStages &&
-          !stage_wait(ptx::smem_u32(&empty_bar[slot]), ((i / kChainStages) - 1) & 1, a.spin_limit)) {
+      // slice i goes to group i % 2; it is that group's k-th slice and uses the k-th slot of its ring
+      const int k = i / kChainGroups, slot = (i % kChainGroups) * ring + k % ring;
+      if (k >= ring && !stage_wait(ptx::smem_u32(&empty_bar[slot]), ((k / ring) - 1) & 1, a.spin_limit)) {
         *abort = 1;
         atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT);
         return;
@@ -480,8 +484,8 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
    for (int i = wi * a.n_slices; i < (wi + 1) * a.n_slices; ++i) {
     if (i % kChainGroups != grp) continue;
     const int slice = i % a.n_slices;
-    const int slot = i % kChainStages;
-    if (!stage_wait(ptx::smem_u32(&full_bar[slot]), (i / kChainStages) & 1, a.spin_limit)) {
+    const int k = i / kChainGroups, slot = grp * ring + k % ring;
+    if (!stage_wait(ptx::smem_u32(&full_bar[slot]), (k / ring) & 1, a.spin_limit)) {
       *abort = 1;
       atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT);
     }
@@ -662,13 +666,17 @@ int launch_score_select(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat
     LRSA_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const int run = (a.BH * g.Wsel + sms - 1) / sms;
     const int runs_per_bh = (g.Wsel + run - 1) / run;
-    const size_t bytes = (size_t)kChainStages * 2 * tok * g.d * sizeof(__nv_bfloat16)   // ring
+    const size_t stage = (size_t)2 * tok * g.d * sizeof(__nv_bfloat16);
+    const size_t rest = (size_t)4 * g.d * sizeof(float) + select_scratch_bytes(g.L) +
+                        (size_t)(kChainGroups * kThreads / 32) * 4 * g.d * sizeof(__nv_bfloat16);
+    const int ring = kChainGroups * kChainMaxRing * stage + rest <= 220 * 1024 ? kChainMaxRing : 2;
+    const size_t bytes = (size_t)kChainGroups * ring * stage                             // rings
                          + (size_t)4 * g.d * sizeof(float)                               // scale / offset
                          + select_scratch_bytes(g.L)
                          + (size_t)(kChainGroups * kThreads / 32) * 4 * g.d * sizeof(__nv_bfloat16);   // min/max reduction
     auto ckern = g.d == 128 ? score_select_chain_kernel<128> : score_select_chain_kernel<64>;
     LRSA_CUDA_CHECK(cudaFuncSetAttribute(ckern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
-    ckern<<<(unsigned)(a.BH * runs_per_bh), kChainThreads, bytes, st>>>(a, run, runs_per_bh);
+    ckern<<<(unsigned)(a.BH * runs_per_bh), kChainThreads, bytes, st>>>(a, run, runs_per_bh, ring);
     LRSA_CUDA_CHECK(cudaGetLastError());
     launch_counter().n++;
     return LRSA_OK;
