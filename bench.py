@@ -184,6 +184,10 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+# DRAM bytes per backward call (dK/dV + dQ kernels) from the ncu summary under profiles/, per workload
+BWD_DRAM_BYTES = {}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -375,10 +379,10 @@ def main():
                         "score_select_frac_of_hbm": kv_bytes(wl) / score_s / 1e9 / peaks["hbm_gbs"]},
         # achieved = effective backward FLOPs (10*d per unmasked pair) / the backward call's CUDA-event time
         # (dK/dV kernel + dQ kernel + ~2 % helpers).  traffic: DRAM bytes of those two kernels in one launch
-        # each (ncu, profiles/lrsa_kernels_cfg2_32k.md: 9115+245 MB and 565+208 MB), known for the 32K workload.
+        # each from an ncu capture; null while the kernels are newer than the last capture.
         "roofline": {"kernel": "lrsa_attn_bwd (lrsa_bwd_dkv_kernel + lrsa_bwd_dq_kernel)", "bound": "tensor",
                      "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
-                     "traffic": 1.0133e10 if wl.name == "cfg2_32k_gqa7_d128" else None,
+                     "traffic": BWD_DRAM_BYTES.get(wl.name),
                      "peak_source": f"{peaks['source']} sustained bf16"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches[0] * args.steps,
     }

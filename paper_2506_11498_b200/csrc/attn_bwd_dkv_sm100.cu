@@ -141,7 +141,7 @@ struct DkvArgs {
 struct DkvBars {
   uint64_t kv_full, acc_done;
   uint64_t ring_full[8], ring_empty[8];
-  uint64_t s_full[2], p_full[2], buf_free[2];
+  uint64_t s_full[2], p_full[2], buf_free[2], red_done[2];
 };
 
 __device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
@@ -162,6 +162,8 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
   __shared__ __align__(16) float st_D[NS][kQRows];
   __shared__ int st_meta[NS][4];             // compact tiles: compact rows visible to the stage's first chunk,
                                              // first column of its second chunk, rows visible to that chunk
+  __shared__ int st_q0[NS], st_hq[NS];       // first query position and query head of the stage (computed once,
+                                             // by the producer: an integer division per thread and tile is costly)
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
 
@@ -191,6 +193,7 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
       mbar_init(smem_u32(&bars.s_full[b]), 2);      // the S^T issuer and the dP^T issuer
       mbar_init(smem_u32(&bars.p_full[b]), 256);    // every softmax thread
       mbar_init(smem_u32(&bars.buf_free[b]), 1);
+      mbar_init(smem_u32(&bars.red_done[b]), 256);  // every softmax thread has read its scratch columns back
     }
     fence_barrier_init();
   }
@@ -242,6 +245,7 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         st_D[slot][lane + 32 * k] = cur[k].y;
         cur[k] = nxt[k];
       }
+      if (lane == 0) { st_q0[slot] = q0; st_hq[slot] = hq; }
       if (lane == 0 && kt.kind == 0) {
         const int cch = (q0 - p.S) / p.L;
         st_meta[slot][0] = p.S + n_hist_windows(cch, p.ndp, p.Wsel) * p.K;
@@ -279,6 +283,7 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
       const int slot = it % NS, b = it & 1;
       ok = mbar_wait_warp(smem_u32(&bars.ring_full[slot]), (it / NS) & 1, abort);
       if (ok && it >= 2) ok = mbar_wait_warp(smem_u32(&bars.buf_free[b]), ((it >> 1) - 1) & 1, abort);
+      if (ok && it >= 2) ok = mbar_wait_warp(smem_u32(&bars.red_done[b]), ((it >> 1) - 1) & 1, abort);
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t d_tmem = tmem + (which == 0 ? Cfg::kColS : Cfg::kColP) + b * kQRows;
@@ -350,8 +355,7 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
       tmem_ld32(P_addr, dp);
       tmem_wait_ld();
       // first query column of this tile that sees this thread's key (64 = none)
-      const int gi = it_begin + it;
-      const int q0 = kt.qb + (gi % kt.nq) * kQRows;
+      const int q0 = st_q0[slot], hq = st_hq[slot];
       int lo;
       if (!key_ok) {
         lo = kQRows;
@@ -400,22 +404,51 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
       tmem_wait_st();
       tc_fence_before_sync();
       mbar_arrive(smem_u32(&bars.p_full[b]));
-      // Off the tensor core's critical path: sum x over the warp's 32 keys by halving exchanges (register
-      // shuffles: shared-memory bandwidth is what the tensor core's operands need); lane l ends with
-      // query column 32*wg + l, which it adds to the per-row accumulator in global memory.
-#pragma unroll
-      for (int m = 16, bit = 16; m >= 1; m >>= 1, bit >>= 1) {
-        const bool up = (lane & bit) != 0;
-#pragma unroll
-        for (int i = 0; i < m; ++i) {
-          const float send = up ? x[i] : x[i + m];
-          const float keep = up ? x[i + m] : x[i];
-          x[i] = keep + __shfl_xor_sync(0xffffffffu, send, bit);
-        }
-      }
+      // Off the tensor core's critical path: sum x over the warp's 32 keys.  The values go through the
+      // upper halves of this warpgroup's own S^T and dP^T columns (free once P^T and dS^T are packed into
+      // the lower halves; the issuers wait for red_done before the buffer is written again) and come back
+      // with the 16-lane x 256-bit load shape, which hands every thread four key rows of eight query
+      // columns; the remaining three levels are register exchanges.  (A full five-level exchange in
+      // registers costs twice the instructions, and shuffles share the shared-memory pipe with the
+      // tensor core's operand reads.)
       {
-        const int hq = hq0 + gi / kt.nq, q = q0 + wg * 32 + lane;
-        if (q < kt.qend) atomicAdd(a.Dacc + (size_t)hq * p.N + q, x[0]);
+        uint32_t xa[16], xb[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) { xa[i] = __float_as_uint(x[i]); xb[i] = __float_as_uint(x[16 + i]); }
+        tmem_st16(S_addr + 16, xa);
+        tmem_st16(P_addr + 16, xb);
+        tmem_wait_st();
+        uint32_t ra0[8], ra1[8], rb0[8], rb1[8];
+        tmem_ld_16x256b_x2(S_addr + 16, ra0);
+        tmem_ld_16x256b_x2(S_addr + 16 + (16u << 16), ra1);
+        tmem_ld_16x256b_x2(P_addr + 16, rb0);
+        tmem_ld_16x256b_x2(P_addr + 16 + (16u << 16), rb1);
+        tmem_wait_ld();
+        tc_fence_before_sync();
+        mbar_arrive(smem_u32(&bars.red_done[b]));
+        float c8[8];   // index 4B + 2j + e: column 16B + 8j + 2(lane%4) + e of the warpgroup's 32
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            c8[2 * j + e] = (__uint_as_float(ra0[4 * j + e]) + __uint_as_float(ra0[4 * j + 2 + e])) +
+                            (__uint_as_float(ra1[4 * j + e]) + __uint_as_float(ra1[4 * j + 2 + e]));
+            c8[4 + 2 * j + e] = (__uint_as_float(rb0[4 * j + e]) + __uint_as_float(rb0[4 * j + 2 + e])) +
+                                (__uint_as_float(rb1[4 * j + e]) + __uint_as_float(rb1[4 * j + 2 + e]));
+          }
+#pragma unroll
+        for (int m = 4, bit = 16; m >= 1; m >>= 1, bit >>= 1) {
+          const bool up = (lane & bit) != 0;
+#pragma unroll
+          for (int i = 0; i < m; ++i) {
+            const float send = up ? c8[i] : c8[i + m];
+            const float keep = up ? c8[i + m] : c8[i];
+            c8[i] = keep + __shfl_xor_sync(0xffffffffu, send, bit);
+          }
+        }
+        const int col = 16 * ((lane >> 4) & 1) + 8 * ((lane >> 3) & 1) + 2 * (lane & 3) + ((lane >> 2) & 1);
+        const int q = q0 + wg * 32 + col;
+        if (q < kt.qend) atomicAdd(a.Dacc + (size_t)hq * p.N + q, c8[0]);
       }
     }
     if (ok) ok = mbar_wait(smem_u32(&bars.acc_done), 0, abort);
