@@ -99,15 +99,48 @@ __host__ __device__ inline int tile_segments(const DkvPlan& p, const KvTile& t) 
   return (p.G * t.nq + kSeg - 1) / kSeg;
 }
 
-// seg_prefix[i] = number of segments of tiles < i   (one block)
-__global__ void dkv_setup_kernel(const DkvPlan p, int* seg_prefix) {
-  for (int i = threadIdx.x; i < p.n_tiles; i += blockDim.x)
-    seg_prefix[i + 1] = tile_segments(p, describe_tile(p, i));
+// Launch order of the (tile, segment) pairs (one block).  Iteration i of a tile is query tile
+// nq-1 - i/G (counted from the last query) of head i%G, so segment s of every compact tile covers the
+// same queries of the same heads.  Compact tiles are therefore issued segment-major: the CTAs that run at
+// the same time then stream the same Q_i / dO_i tiles and share them through L2 instead of fetching
+// them from DRAM once per key tile.  Dense tiles (short lists, neighbours already overlap) follow in
+// position order.  seg_cnt: scratch of n_tiles + 1 ints; seg_map[x] = (tile, segment of the tile).
+constexpr int kMaxSegsPerTile = 2048;
+__global__ void dkv_setup_kernel(const DkvPlan p, int* seg_cnt, int2* seg_map) {
+  __shared__ int off[kMaxSegsPerTile + 1];   // off[s] = pairs of compact tiles with a segment index below s
+  __shared__ int s_mode;
+  for (int i = threadIdx.x; i < p.n_tiles; i += blockDim.x) seg_cnt[i] = tile_segments(p, describe_tile(p, i));
   __syncthreads();
   if (threadIdx.x == 0) {
-    int acc = 0;
-    seg_prefix[0] = 0;
-    for (int i = 1; i <= p.n_tiles; ++i) { acc += seg_prefix[i]; seg_prefix[i] = acc; }
+    // segment-major order needs the compact tiles' segment counts to be non-increasing (later rows are
+    // seen by later chunks only) and few enough for the table; otherwise keep tile-major order
+    bool mono = p.n_cmp > 0 && seg_cnt[0] <= kMaxSegsPerTile;
+    for (int c = 1; c < p.n_cmp && mono; ++c) mono = seg_cnt[c] <= seg_cnt[c - 1];
+    int total = 0;
+    if (mono) {
+      int c = p.n_cmp;   // tiles [0, c) have more than s segments
+      const int maxs = seg_cnt[0];
+      for (int sgm = 0; sgm < maxs; ++sgm) {
+        while (c > 0 && seg_cnt[c - 1] <= sgm) --c;
+        off[sgm] = total;
+        total += c;
+      }
+    } else {
+      for (int c = 0; c < p.n_cmp; ++c) {
+        for (int sgm = 0; sgm < seg_cnt[c]; ++sgm) seg_map[total + sgm] = make_int2(c, sgm);
+        total += seg_cnt[c];
+      }
+    }
+    s_mode = mono ? 1 : 0;
+    for (int t = p.n_cmp; t < p.n_tiles; ++t) {   // dense tiles, position order
+      for (int sgm = 0; sgm < seg_cnt[t]; ++sgm) seg_map[total + sgm] = make_int2(t, sgm);
+      total += seg_cnt[t];
+    }
+  }
+  __syncthreads();
+  if (s_mode) {
+    for (int c = threadIdx.x; c < p.n_cmp; c += blockDim.x)
+      for (int sgm = 0; sgm < seg_cnt[c]; ++sgm) seg_map[off[sgm] + c] = make_int2(c, sgm);
   }
 }
 
@@ -130,7 +163,7 @@ struct DkvArgs {
   int BHkv, Hq, Hkv, total_segs;
   const float2* stats;   // per query row: (-LSE * log2(e), D~ = rowsum(dO * O) from the bf16 O)
   float* Dacc;           // [B*Hq][N], zeroed: receives sum_j P_tj dP_tj, the accurate D for the dQ kernel
-  const int* seg_prefix;
+  const int2* seg_map;   // launch order: (tile, segment of the tile)
   float* dKf;   // [BHkv][N + Rc][D] fp32, zeroed
   float* dVf;
   int rows_ws;  // N + Rc
@@ -174,13 +207,9 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
   // ---- which tile, which segment ----
   const DkvPlan& p = a.plan;
   const int bh_kv = blockIdx.x % a.BHkv, seg = blockIdx.x / a.BHkv;
-  int lo_t = 0, hi_t = p.n_tiles;   // last tile with seg_prefix[tile] <= seg
-  while (hi_t - lo_t > 1) {
-    const int mid = (lo_t + hi_t) >> 1;
-    if (a.seg_prefix[mid] <= seg) lo_t = mid; else hi_t = mid;
-  }
-  const KvTile kt = describe_tile(p, lo_t);
-  const int it_begin = (seg - a.seg_prefix[lo_t]) * kSeg;
+  const int2 ts = a.seg_map[seg];
+  const KvTile kt = describe_tile(p, ts.x);
+  const int it_begin = ts.y * kSeg;
   const int n = min(kSeg, p.G * kt.nq - it_begin);
   const int hq0 = (bh_kv / a.Hkv) * a.Hq + (bh_kv % a.Hkv) * p.G;   // first query head of the group
 
@@ -220,9 +249,10 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     int it = 0;
     // per-row statistics of a stage are fetched one stage ahead, so that their latency overlaps the
     // wait for a free slot instead of adding to it
-    auto fetch = [&](int i, float2 (&v)[kQRows / 32]) {
-      const int gi = it_begin + i;
-      const int hq = hq0 + gi / kt.nq, q0 = kt.qb + (gi % kt.nq) * kQRows;
+    // iteration gi: query tile nq-1 - gi/G (from the last query backwards) of head gi % G
+    int qt = kt.nq - 1 - it_begin / p.G, hd = it_begin % p.G;
+    auto fetch = [&](int qt_, int hd_, float2 (&v)[kQRows / 32]) {
+      const int hq = hq0 + hd_, q0 = kt.qb + qt_ * kQRows;
 #pragma unroll
       for (int k = 0; k < kQRows / 32; ++k) {
         const int q = q0 + lane + 32 * k;
@@ -230,15 +260,16 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
       }
     };
     float2 cur[kQRows / 32], nxt[kQRows / 32];
-    if (n > 0) fetch(0, cur);
+    if (n > 0) fetch(qt, hd, cur);
     for (; it < n; ++it) {
       const int slot = it % NS, use = it / NS;
-      if (it + 1 < n) fetch(it + 1, nxt);
+      int qt_n = qt, hd_n = hd + 1;
+      if (hd_n == p.G) { hd_n = 0; --qt_n; }
+      if (it + 1 < n) fetch(qt_n, hd_n, nxt);
       if (use > 0 && lane == 0) ok = mbar_wait(smem_u32(&bars.ring_empty[slot]), (use - 1) & 1, abort);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
-      const int gi = it_begin + it;
-      const int hq = hq0 + gi / kt.nq, q0 = kt.qb + (gi % kt.nq) * kQRows;
+      const int hq = hq0 + hd, q0 = kt.qb + qt * kQRows;
 #pragma unroll
       for (int k = 0; k < kQRows / 32; ++k) {
         st_nl2[slot][lane + 32 * k] = cur[k].x;
@@ -262,6 +293,7 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
           tma_load_3d(dst + Cfg::kQTileBytes + h * Cfg::kQSubBytes, &mapdO, h * 64, q0, hq, full);
         }
       }
+      qt = qt_n; hd = hd_n;
     }
     if (!ok && lane == 0) {
       for (int back = 1; back <= NS && back <= it; ++back) {
@@ -513,9 +545,17 @@ __global__ void convert_dkv_kernel(const float* __restrict__ dKf, const float* _
 
 }  // namespace
 
+static int dkv_total_segs(const DkvPlan& p) {
+  int total = 0;
+  for (int i = 0; i < p.n_tiles; ++i) total += tile_segments(p, describe_tile(p, i));
+  return total;
+}
+
+// Layout: [segment counts: n_tiles + 1 ints][launch order: total_segs int2][dK fp32][dV fp32]
 size_t dkv_ws_bytes(const Geom& g, size_t* prefix_bytes) {
   const DkvPlan p = make_dkv_plan(g);
-  const size_t pre = align_up((size_t)(p.n_tiles + 1) * sizeof(int), 1024);
+  const size_t cnt = align_up((size_t)(p.n_tiles + 1) * sizeof(int), 1024);
+  const size_t pre = cnt + align_up((size_t)(dkv_total_segs(p) + 1) * sizeof(int2), 1024);
   if (prefix_bytes) *prefix_bytes = pre;
   const size_t acc = align_up((size_t)g.B * g.Hkv * (g.N + g.Rc) * g.d * sizeof(float), 1024);
   return pre + 2 * acc;
@@ -546,16 +586,16 @@ int launch_bwd_dkv_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloa
   const size_t total = dkv_ws_bytes(g, &pre);
   unsigned char* base = static_cast<unsigned char*>(ws_dkv);
   const size_t acc = (total - pre) / 2;
-  int* seg_prefix = reinterpret_cast<int*>(base);
+  int* seg_cnt = reinterpret_cast<int*>(base);
+  int2* seg_map = reinterpret_cast<int2*>(base + align_up((size_t)(p.n_tiles + 1) * sizeof(int), 1024));
   float* dKf = reinterpret_cast<float*>(base + pre);
   float* dVf = reinterpret_cast<float*>(base + pre + acc);
   LRSA_CUDA_CHECK(cudaMemsetAsync(base + pre, 0, 2 * acc, st));
   launch_counter().n++;
-  dkv_setup_kernel<<<1, 256, 0, st>>>(p, seg_prefix);
+  dkv_setup_kernel<<<1, 256, 0, st>>>(p, seg_cnt, seg_map);
   LRSA_CUDA_CHECK(cudaGetLastError());
   launch_counter().n++;
-  int total_segs = 0;
-  for (int i = 0; i < p.n_tiles; ++i) total_segs += tile_segments(p, describe_tile(p, i));
+  const int total_segs = dkv_total_segs(p);
 
   CUtensorMap m[6];
   const long long rc = g.Rc > 0 ? g.Rc : 1;
@@ -568,7 +608,7 @@ int launch_bwd_dkv_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloa
   if (r != LRSA_OK) return r;
   DkvArgs a;
   a.plan = p; a.BHkv = g.B * g.Hkv; a.Hq = g.Hq; a.Hkv = g.Hkv; a.total_segs = total_segs;
-  a.stats = stats; a.Dacc = Dacc; a.seg_prefix = seg_prefix; a.dKf = dKf; a.dVf = dVf; a.rows_ws = g.N + g.Rc;
+  a.stats = stats; a.Dacc = Dacc; a.seg_map = seg_map; a.dKf = dKf; a.dVf = dVf; a.rows_ws = g.N + g.Rc;
   a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f; a.status = status;
   r = g.d == 128 ? launch_dkv_t<128>(g, a, m, st) : launch_dkv_t<64>(g, a, m, st);
   if (r != LRSA_OK) return r;
