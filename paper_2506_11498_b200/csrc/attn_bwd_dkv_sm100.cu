@@ -6,7 +6,7 @@
 //   dense tiles   : original positions of one window (or of the sink region / the tail); seen
 //                   causally by the queries from the diagonal to the end of the last chunk that
 //                   still sees that window uncompressed
-// A CTA takes one tile and a segment of its (query head of the group, 64-row query tile) list:
+// A CTA takes one tile and a segment of its (64-row query tile, query head of the group) list:
 //   S^T  = K_j Q_i^T     (smem x smem -> TMEM, keys on lanes)     P^T  = exp2(S^T*c - LSE_i*log2e)
 //   dP^T = V_j dO_i^T    (smem x smem -> TMEM)                    dS^T = P^T * (dP^T - D_i)
 //   dV  += P^T dO_i      (TMEM x smem -> TMEM)
@@ -14,9 +14,12 @@
 // P^T and dS^T are written back over S^T and dP^T as packed bf16; both are double-buffered so the
 // tensor core computes the next S^T/dP^T while the current pair is in the softmax, on which both
 // warpgroups work (32 query columns each).  Warps: 0 producer, 1-3 tensor-core issuers (S^T, dP^T,
-// dV/dK), 4-11 softmax and epilogue.  The softmax warps also sum P^T * dP^T over the keys and add it to
-// a per-query-row accumulator: D_i = sum_j P_ij dP_ij, the accurate replacement of rowsum(dO * O)
-// that the dQ kernel (which runs afterwards) needs.  At the end
+// dV/dK), 4-11 softmax and epilogue.  The softmax warps also sum P^T * dP^T over the keys (through
+// spare tensor-memory columns and a transposing load shape) and add it to a per-query-row accumulator:
+// D_i = sum_j P_ij dP_ij, the accurate replacement of rowsum(dO * O) that the dQ kernel (which runs
+// afterwards) needs.  The list of a tile runs from the last query tile backwards with the heads
+// innermost, and compact tiles are launched segment by segment, so that the CTAs resident at one time
+// read the same Q_i / dO_i tiles (L2 hits instead of one DRAM pass per key tile).  At the end
 // the accumulators are added (fp32 atomics) to a zeroed workspace indexed by original position
 // (dense tiles) or by compact row (compact tiles); two small kernels then fold the compact rows
 // onto their original positions and convert to bf16.
@@ -108,7 +111,8 @@ __host__ __device__ inline int tile_segments(const DkvPlan& p, const KvTile& t) 
 constexpr int kMaxSegsPerTile = 2048;
 __global__ void dkv_setup_kernel(const DkvPlan p, int* seg_cnt, int2* seg_map) {
   __shared__ int off[kMaxSegsPerTile + 1];   // off[s] = pairs of compact tiles with a segment index below s
-  __shared__ int s_mode;
+  __shared__ int s_mode, s_cmp_total;
+  __shared__ int run_sum[256];   // blockDim.x = 256
   for (int i = threadIdx.x; i < p.n_tiles; i += blockDim.x) seg_cnt[i] = tile_segments(p, describe_tile(p, i));
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -132,12 +136,27 @@ __global__ void dkv_setup_kernel(const DkvPlan p, int* seg_cnt, int2* seg_map) {
       }
     }
     s_mode = mono ? 1 : 0;
-    for (int t = p.n_cmp; t < p.n_tiles; ++t) {   // dense tiles, position order
-      for (int sgm = 0; sgm < seg_cnt[t]; ++sgm) seg_map[total + sgm] = make_int2(t, sgm);
-      total += seg_cnt[t];
-    }
+    s_cmp_total = total;
+  }
+  // dense tiles, position order: every thread takes a run of consecutive tiles
+  const int nd = p.n_tiles - p.n_cmp, per = (nd + (int)blockDim.x - 1) / (int)blockDim.x;
+  const int d_lo = min(p.n_tiles, p.n_cmp + (int)threadIdx.x * per), d_hi = min(p.n_tiles, d_lo + per);
+  int mine = 0;
+  for (int t = d_lo; t < d_hi; ++t) mine += seg_cnt[t];
+  run_sum[threadIdx.x] = mine;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int acc = s_cmp_total;
+    for (int i = 0; i < (int)blockDim.x; ++i) { const int v = run_sum[i]; run_sum[i] = acc; acc += v; }
   }
   __syncthreads();
+  {
+    int pos = run_sum[threadIdx.x];
+    for (int t = d_lo; t < d_hi; ++t) {
+      for (int sgm = 0; sgm < seg_cnt[t]; ++sgm) seg_map[pos + sgm] = make_int2(t, sgm);
+      pos += seg_cnt[t];
+    }
+  }
   if (s_mode) {
     for (int c = threadIdx.x; c < p.n_cmp; c += blockDim.x)
       for (int sgm = 0; sgm < seg_cnt[c]; ++sgm) seg_map[off[sgm] + c] = make_int2(c, sgm);

@@ -303,10 +303,21 @@ __global__ void bwd_prep_kernel(const __nv_bfloat16* __restrict__ O, const __nv_
   if (row >= rows) return;
   const int lane = threadIdx.x & 31;
   float acc = 0.f;
-  for (int c = lane * 2; c < d; c += 64) {
-    const __nv_bfloat162 o = *reinterpret_cast<const __nv_bfloat162*>(O + row * d + c);
-    const __nv_bfloat162 g = *reinterpret_cast<const __nv_bfloat162*>(dO + row * d + c);
-    acc += __bfloat162float(o.x) * __bfloat162float(g.x) + __bfloat162float(o.y) * __bfloat162float(g.y);
+  if ((d & 127) == 0) {   // 8 bytes per lane and load: a 128-element row in one load per tensor
+    for (int c = lane * 4; c < d; c += 128) {
+      const uint2 o = *reinterpret_cast<const uint2*>(O + row * d + c);
+      const uint2 g = *reinterpret_cast<const uint2*>(dO + row * d + c);
+      acc = fmaf(__uint_as_float(o.x << 16), __uint_as_float(g.x << 16), acc);
+      acc = fmaf(__uint_as_float(o.x & 0xffff0000u), __uint_as_float(g.x & 0xffff0000u), acc);
+      acc = fmaf(__uint_as_float(o.y << 16), __uint_as_float(g.y << 16), acc);
+      acc = fmaf(__uint_as_float(o.y & 0xffff0000u), __uint_as_float(g.y & 0xffff0000u), acc);
+    }
+  } else {
+    for (int c = lane * 2; c < d; c += 64) {
+      const __nv_bfloat162 o = *reinterpret_cast<const __nv_bfloat162*>(O + row * d + c);
+      const __nv_bfloat162 g = *reinterpret_cast<const __nv_bfloat162*>(dO + row * d + c);
+      acc += __bfloat162float(o.x) * __bfloat162float(g.x) + __bfloat162float(o.y) * __bfloat162float(g.y);
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
