@@ -435,20 +435,28 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
       const float4* Dv = reinterpret_cast<const float4*>(st_D[slot] + wg * 32);
       uint32_t pp[16], ds[16];
       float x[32];   // P * dP, whose sum over the keys is the accurate D of the query column
+      {
+        // packed fp32 pairs: one issue slot for two elements of every multiply-add below
+        const uint64_t c2 = f2_pack(c, c);
 #pragma unroll
-      for (int v = 0; v < 8; ++v) {
-        const float4 nl = nl2v[v], dd = Dv[v];
-        const float p0 = ex2(fmaf(__uint_as_float(s[4 * v + 0]), c, nl.x));
-        const float p1 = ex2(fmaf(__uint_as_float(s[4 * v + 1]), c, nl.y));
-        const float p2 = ex2(fmaf(__uint_as_float(s[4 * v + 2]), c, nl.z));
-        const float p3 = ex2(fmaf(__uint_as_float(s[4 * v + 3]), c, nl.w));
-        const float g0 = __uint_as_float(dp[4 * v + 0]), g1 = __uint_as_float(dp[4 * v + 1]);
-        const float g2 = __uint_as_float(dp[4 * v + 2]), g3 = __uint_as_float(dp[4 * v + 3]);
-        pp[2 * v] = pack_bf16(p0, p1);
-        pp[2 * v + 1] = pack_bf16(p2, p3);
-        x[4 * v + 0] = p0 * g0; x[4 * v + 1] = p1 * g1; x[4 * v + 2] = p2 * g2; x[4 * v + 3] = p3 * g3;
-        ds[2 * v] = pack_bf16(fmaf(-p0, dd.x, x[4 * v + 0]), fmaf(-p1, dd.y, x[4 * v + 1]));
-        ds[2 * v + 1] = pack_bf16(fmaf(-p2, dd.z, x[4 * v + 2]), fmaf(-p3, dd.w, x[4 * v + 3]));
+        for (int v = 0; v < 8; ++v) {
+          const float4 nl = nl2v[v], dd = Dv[v];
+          float a0, a1, a2, a3, d0, d1, d2, d3;
+          f2_unpack(f2_fma(f2_pack(__uint_as_float(s[4 * v + 0]), __uint_as_float(s[4 * v + 1])), c2, f2_pack(nl.x, nl.y)), a0, a1);
+          f2_unpack(f2_fma(f2_pack(__uint_as_float(s[4 * v + 2]), __uint_as_float(s[4 * v + 3])), c2, f2_pack(nl.z, nl.w)), a2, a3);
+          const float p0 = ex2(a0), p1 = ex2(a1), p2 = ex2(a2), p3 = ex2(a3);
+          pp[2 * v] = pack_bf16(p0, p1);
+          pp[2 * v + 1] = pack_bf16(p2, p3);
+          const uint64_t p01 = f2_pack(p0, p1), p23 = f2_pack(p2, p3);
+          const uint64_t x01 = f2_mul(p01, f2_pack(__uint_as_float(dp[4 * v + 0]), __uint_as_float(dp[4 * v + 1])));
+          const uint64_t x23 = f2_mul(p23, f2_pack(__uint_as_float(dp[4 * v + 2]), __uint_as_float(dp[4 * v + 3])));
+          f2_unpack(x01, x[4 * v + 0], x[4 * v + 1]);
+          f2_unpack(x23, x[4 * v + 2], x[4 * v + 3]);
+          f2_unpack(f2_fma(p01, f2_pack(-dd.x, -dd.y), x01), d0, d1);   // dS = P dP - P D
+          f2_unpack(f2_fma(p23, f2_pack(-dd.z, -dd.w), x23), d2, d3);
+          ds[2 * v] = pack_bf16(d0, d1);
+          ds[2 * v + 1] = pack_bf16(d2, d3);
+        }
       }
       tmem_st16(S_addr, pp);   // over the first half of this warpgroup's own columns
       tmem_st16(P_addr, ds);

@@ -243,14 +243,23 @@ lrsa_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
           if (i >= limit) s[i] = 0xff800000u;
       }
       uint32_t ds[16];
-      float r0 = 0.f, r1 = 0.f;
+      float r0, r1;
+      {
+        // packed fp32 pairs: one issue slot for two elements of the scale-and-shift, of dP - D, of the
+        // product and of the row sum of the rounded dS
+        const uint64_t c2 = f2_pack(c, c), nl22 = f2_pack(nl2, nl2), nD2 = f2_pack(-Dt, -Dt);
+        uint64_t r2 = f2_pack(0.f, 0.f);
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const float p0 = ex2(fmaf(__uint_as_float(s[2 * i]), c, nl2));
-        const float p1 = ex2(fmaf(__uint_as_float(s[2 * i + 1]), c, nl2));
-        ds[i] = pack_bf16(p0 * (__uint_as_float(dp[2 * i]) - Dt), p1 * (__uint_as_float(dp[2 * i + 1]) - Dt));
-        r0 += __uint_as_float(ds[i] << 16);
-        r1 += __uint_as_float(ds[i] & 0xffff0000u);
+        for (int i = 0; i < 16; ++i) {
+          float x0, x1, d0, d1;
+          f2_unpack(f2_fma(f2_pack(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), c2, nl22), x0, x1);
+          const float p0 = ex2(x0), p1 = ex2(x1);
+          const uint64_t g2 = f2_add(f2_pack(__uint_as_float(dp[2 * i]), __uint_as_float(dp[2 * i + 1])), nD2);
+          f2_unpack(f2_mul(f2_pack(p0, p1), g2), d0, d1);
+          ds[i] = pack_bf16(d0, d1);
+          r2 = f2_add(r2, f2_pack(__uint_as_float(ds[i] << 16), __uint_as_float(ds[i] & 0xffff0000u)));
+        }
+        f2_unpack(r2, r0, r1);
       }
       rsum += r0 + r1;
       tmem_st16(S_addr, ds);   // over the first half of this warpgroup's own S columns
