@@ -200,10 +200,6 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     tc_fence_before_sync();
     mbar_arrive(smem_u32(&bars.qt_ready));   // also when the wait gave up: the issuers then see abort
     float m = -INFINITY, l = 0.f;
-    // Start the second warpgroup about half a tile late: the two then stay out of phase (nothing
-    // re-aligns them while the S tiles arrive ahead of the softmax), so one warpgroup's exponentials
-    // keep the MUFU pipe busy while the other loads S and takes row maxima.
-    if (half == 1 && n > 1) __nanosleep(400);
     for (int j = 0; j < n && ok; ++j) {
       const int b = j & 1;
       ok = mbar_wait(smem_u32(&bars.s_full[b]), (j >> 1) & 1, abort);
