@@ -479,6 +479,27 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
    const int w = w_b - wi;
    const bool scoring = wi > 0;          // the first window streamed is a reference only
    const bool want_stats = w > w_a;      // its statistics serve the next window of the run
+   // scale and offset (Eq. 6) of this thread's eight channels, as packed pairs: [tensor][sa, sb][pair]
+   uint64_t sab2[2][2][4];
+   if (scoring) {
+#pragma unroll
+     for (int z = 0; z < 2; ++z)
+#pragma unroll
+       for (int m = 0; m < 2; ++m)
+#pragma unroll
+         for (int h = 0; h < 2; ++h) {
+           const float4 v = *reinterpret_cast<const float4*>(sasb + (z * 2 + m) * D + chunk * 8 + h * 4);
+           sab2[z][m][2 * h] = ptx::f2_pack(v.x, v.y);
+           sab2[z][m][2 * h + 1] = ptx::f2_pack(v.z, v.w);
+         }
+   } else {
+#pragma unroll
+     for (int z = 0; z < 2; ++z)
+#pragma unroll
+       for (int m = 0; m < 2; ++m)
+#pragma unroll
+         for (int j = 0; j < 4; ++j) sab2[z][m][j] = 0ull;
+   }
 #pragma unroll
    for (int j = 0; j < 4; ++j) { st[0][0][j] = st[1][0][j] = PINF; st[0][1][j] = st[1][1][j] = NINF; }
    for (int i = wi * a.n_slices; i < (wi + 1) * a.n_slices; ++i) {
@@ -521,40 +542,69 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
       }
     }
     if (scoring) {
-      // Eq. 6 with the statistics of window w+1 (z' = x*sa + sb = zbar - 1/2) and the per-token Std of Eq. 7
+      // Eq. 6 with the statistics of window w+1 (z' = x*sa + sb = zbar - 1/2) and the per-token Std of
+      // Eq. 7.  Arithmetic on packed fp32 pairs; sa/sb of this thread's eight channels live in registers
+      // for the whole window (sab2, loaded below the window loop's head).
+      float part[2 * kSteps][2];   // [tensor * kSteps + step][sum, sum of squares] over this thread's 8 channels
 #pragma unroll
       for (int z = 0; z < 2; ++z) {
-        float sa[8], sb[8];
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const float4 va = *reinterpret_cast<const float4*>(sasb + (z * 2 + 0) * D + chunk * 8 + h * 4);
-          const float4 vb = *reinterpret_cast<const float4*>(sasb + (z * 2 + 1) * D + chunk * 8 + h * 4);
-          sa[h * 4 + 0] = va.x; sa[h * 4 + 1] = va.y; sa[h * 4 + 2] = va.z; sa[h * 4 + 3] = va.w;
-          sb[h * 4 + 0] = vb.x; sb[h * 4 + 1] = vb.y; sb[h * 4 + 2] = vb.z; sb[h * 4 + 3] = vb.w;
-        }
-        float* out = z == 0 ? sk : sv;
 #pragma unroll
         for (int s = 0; s < kSteps; ++s) {
           const uint4 q = z == 0 ? kq[s] : vq[s];
           const uint32_t pk[4] = {q.x, q.y, q.z, q.w};
-          float sum = 0.f, sq = 0.f;
+          uint64_t sum2 = 0ull, sq2 = 0ull;   // (+0, +0)
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const float z0 = fmaf(bf_lo(pk[j]), sa[2 * j], sb[2 * j]);
-            const float z1 = fmaf(bf_hi(pk[j]), sa[2 * j + 1], sb[2 * j + 1]);
-            sum += z0 + z1;
-            sq = fmaf(z0, z0, sq);
-            sq = fmaf(z1, z1, sq);
+            const uint64_t z2 = ptx::f2_fma(ptx::f2_pack(bf_lo(pk[j]), bf_hi(pk[j])), sab2[z][0][j], sab2[z][1][j]);
+            sum2 = ptx::f2_add(sum2, z2);
+            sq2 = ptx::f2_fma(z2, z2, sq2);
           }
+          float s0, s1, q0, q1;
+          ptx::f2_unpack(sum2, s0, s1);
+          ptx::f2_unpack(sq2, q0, q1);
+          part[z * kSteps + s][0] = s0 + s1;
+          part[z * kSteps + s][1] = q0 + q1;
+        }
+      }
+      // Sum over the LPR lanes of a row.  Halving exchange: at every level a lane keeps half of its
+      // entries and hands the other half to its partner, so 2*kSteps entries cost 2*(2*kSteps - 1)
+      // shuffles instead of 2*kSteps*log2(LPR)*2; levels left over once one entry remains are plain
+      // butterflies.  The lane ends with entry e(chunk) complete.
+      int ent = 0;   // index of the entry this lane ends up with
+      {
+        int m = 2 * kSteps;   // entries still held
 #pragma unroll
-          for (int o = LPR / 2; o > 0; o >>= 1) {
-            sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            sq += __shfl_xor_sync(0xffffffffu, sq, o);
+        for (int bit = LPR / 2; bit >= 1; bit >>= 1) {
+          if (m > 1) {
+            m >>= 1;
+            const bool up = (chunk & bit) != 0;
+#pragma unroll
+            for (int e = 0; e < kSteps; ++e) {   // kSteps >= m at every level
+              if (e < m) {
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                  const float send = up ? part[e][c] : part[e + m][c];
+                  const float keep = up ? part[e + m][c] : part[e][c];
+                  part[e][c] = keep + __shfl_xor_sync(0xffffffffu, send, bit);
+                }
+              }
+            }
+            ent += up ? m : 0;
+          } else {
+            part[0][0] += __shfl_xor_sync(0xffffffffu, part[0][0], bit);
+            part[0][1] += __shfl_xor_sync(0xffffffffu, part[0][1], bit);
           }
-          if (chunk == 0 && valid[s]) {
-            const float var = (sq - sum * sum * (1.0f / D)) * inv_dof;
-            out[slice * TOK + s * RPS + row] = sqrtf(fmaxf(var, 0.f));
-          }
+        }
+      }
+      {
+        const int z = ent / kSteps, st_ = ent % kSteps;
+        // lanes that differ only in the bits of the plain butterfly levels hold the same entry: one writes
+        constexpr int kDup = LPR / (2 * kSteps) > 1 ? LPR / (2 * kSteps) : 1;
+        const bool writer = (chunk & (kDup - 1)) == 0;
+        const int tkn = slice * TOK + st_ * RPS + row;
+        if (writer && tkn < a.L) {
+          const float var = (part[0][1] - part[0][0] * part[0][0] * (1.0f / D)) * inv_dof;
+          (z == 0 ? sk : sv)[tkn] = sqrtf(fmaxf(var, 0.f));
         }
       }
     }
