@@ -122,18 +122,36 @@ __device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* 
   for (int i = 0; i < 8; ++i) { ek += red[i]; ev += red[8 + i]; }
   // Eq. 8
   float* gs = a.score ? a.score + (size_t)(bh * a.Wsel + w) * L : nullptr;
+  uint32_t kmin = 0xffffffffu, kmax = 0u;   // range of the keys (scores are positive: bit order = value order)
   for (int i = tid; i < L; i += kThreads) {
     const float s = sk[i] / ek + sv[i] / ev;
     sk[i] = s;
     if (gs) gs[i] = s;
+    kmin = min(kmin, __float_as_uint(s));
+    kmax = max(kmax, __float_as_uint(s));
   }
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  scoring_warps_sync();   // also: every read of red[] above is done
+  uint32_t* kred = reinterpret_cast<uint32_t*>(red);
+  if (lane == 0) { kred[warp] = kmin; kred[8 + warp] = kmax; }
   scoring_warps_sync();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { kmin = min(kmin, kred[i]); kmax = max(kmax, kred[8 + i]); }
 
   // radix select of the K-th largest score; scores are positive, so bit order = value order
+  // The keys of a window share their leading bits (the scores of one window lie within a small factor of
+  // each other): those bits are fixed at once, and the 8-bit passes start at the highest bit in which two
+  // keys differ.  (A pass over shared bits would also send every key to one histogram bin: a thousand
+  // serialised shared-memory atomics.)
   const uint32_t* key = reinterpret_cast<const uint32_t*>(sk);
-  uint32_t prefix = 0, mask = 0;
+  const uint32_t diff = kmin ^ kmax;
+  const int top = diff ? 31 - __clz(diff) : -1;                  // highest differing bit, -1: all keys equal
+  uint32_t mask = top >= 31 ? 0u : ~((2u << (top < 0 ? 0 : top)) - 1u);
+  if (top < 0) mask = 0xffffffffu;
+  uint32_t prefix = kmax & mask;
   int remaining = a.Kk;
-  for (int shift = 24; shift >= 0; shift -= 8) {
+  for (int shift = top < 0 ? -1 : max(top - 7, 0); shift >= 0; shift = shift == 0 ? -1 : max(shift - 8, 0)) {
     hist[tid] = 0;
     scoring_warps_sync();
     for (int i = tid; i < L; i += kThreads) {
@@ -169,37 +187,41 @@ __device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* 
   const uint32_t kth = prefix;    // K-th largest key
   const int need_eq = remaining;  // how many keys equal to it are kept (lowest positions first)
 
-  // emit kept positions in ascending order
+  // emit kept positions in ascending order: every thread takes a run of consecutive tokens, one block
+  // scan gives the number of kept tokens before the run
   int32_t* out = a.idx + (size_t)(bh * a.Wsel + w) * a.Kk;
-  int base_gt = 0, base_eq = 0;
-  int* wtot = ibuf;  // 8 warp totals
-  for (int i0 = 0; i0 < L; i0 += kThreads) {
-    const int i = i0 + tid;
-    const uint32_t k = i < L ? key[i] : 0u;
-    const int gt = (i < L && k > kth) ? 1 : 0, eq = (i < L && k == kth) ? 1 : 0;
-    const int packed = gt | (eq << 16);
-    int incl = packed;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int n = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += n;
-    }
-    if (lane == 31) wtot[warp] = incl;
-    scoring_warps_sync();
-    int excl = incl - packed, all = 0;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int t = wtot[j];
-      if (j < warp) excl += t;
-      all += t;
-    }
-    const int gt_before = base_gt + (excl & 0xffff), eq_before = base_eq + (excl >> 16);
-    if (gt || (eq && eq_before < need_eq))
-      out[gt_before + min(eq_before, need_eq)] = a.S + w * L + i;
-    base_gt += all & 0xffff;
-    base_eq += all >> 16;
-    scoring_warps_sync();
+  const int per = (L + kThreads - 1) / kThreads;
+  const int i_lo = min(L, tid * per), i_hi = min(L, i_lo + per);
+  int packed = 0;   // tokens above the K-th score | tokens equal to it << 16
+  for (int i = i_lo; i < i_hi; ++i) {
+    const uint32_t k = key[i];
+    packed += (k > kth ? 1 : 0) | (k == kth ? 1 << 16 : 0);
   }
+  int incl = packed;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += n;
+  }
+  int* wtot = ibuf;  // 8 warp totals (ibuf's last readers passed the barrier that ended the last pass)
+  if (lane == 31) wtot[warp] = incl;
+  scoring_warps_sync();
+  int excl = incl - packed;
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    if (j < warp) excl += wtot[j];
+  int gt_before = excl & 0xffff, eq_before = excl >> 16;
+  for (int i = i_lo; i < i_hi; ++i) {
+    const uint32_t k = key[i];
+    if (k > kth) {
+      out[gt_before + min(eq_before, need_eq)] = a.S + w * L + i;
+      ++gt_before;
+    } else if (k == kth) {
+      if (eq_before < need_eq) out[gt_before + eq_before] = a.S + w * L + i;
+      ++eq_before;
+    }
+  }
+  scoring_warps_sync();   // sk and ibuf may be reused by the caller
 }
 
 template <int D>
