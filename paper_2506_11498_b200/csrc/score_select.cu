@@ -528,12 +528,16 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
     if (i % kChainGroups != grp) continue;
     const int slice = i % a.n_slices;
     const int k = i / kChainGroups, slot = grp * ring + k % ring;
-    if (!stage_wait(ptx::smem_u32(&full_bar[slot]), (k / ring) & 1, a.spin_limit)) {
+    // One barrier per slice: a warp whose wait ran out skips the arithmetic (warp-uniform, the
+    // arithmetic shuffles), raises the flag and still meets the group at the barrier below, after
+    // which every thread of the group reads the same verdict.
+    bool got = stage_wait(ptx::smem_u32(&full_bar[slot]), (k / ring) & 1, a.spin_limit);
+    got = __all_sync(0xffffffffu, got);
+    if (!got) {
       *abort = 1;
       atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT);
     }
-    group_sync(grp);
-    if (*abort) break;   // the same verdict for every thread of the group: it was written before the barrier
+    if (__all_sync(0xffffffffu, got && !*abort)) {
     const unsigned char* stage = smem + slot * kStageBytes;
     // this thread's rows of the slice: kSteps rows of K and of V, 16 bytes (8 channels) each
     uint4 kq[kSteps], vq[kSteps];
@@ -630,7 +634,9 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
         }
       }
     }
+    }
     group_sync(grp);   // every read of the stage by this group is done
+    if (*abort) break;   // written before the barrier by whichever thread gave up
     if (gt == 0) ptx::mbar_arrive(ptx::smem_u32(&empty_bar[slot]));
    }
 
