@@ -461,16 +461,19 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
   if (warp == kChainGroups * kThreads / 32) {
     // ---------------- producer ----------------
     if (lane != 0) return;
+    // slice i goes to group i % 2; it is that group's k-th slice and uses slot k % ring of its ring in
+    // that slot's (k / ring)-th use.  All counters advance without divisions: one thread feeds the SM.
+    static_assert(kChainGroups == 2, "slot bookkeeping below");
+    int kr[2] = {0, 0}, use[2] = {0, 0};   // per group: k % ring and k / ring of its next slice
+    int w = w_b, slice = 0;
     for (int i = 0; i < n_it; ++i) {
-      // slice i goes to group i % 2; it is that group's k-th slice and uses the k-th slot of its ring
-      const int k = i / kChainGroups, slot = (i % kChainGroups) * ring + k % ring;
-      if (k >= ring && !stage_wait(ptx::smem_u32(&empty_bar[slot]), ((k / ring) - 1) & 1, a.spin_limit)) {
+      const int g = i & 1, slot = g * ring + kr[g];
+      if (use[g] > 0 && !stage_wait(ptx::smem_u32(&empty_bar[slot]), (use[g] - 1) & 1, a.spin_limit)) {
         *abort = 1;
         atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT);
         return;
       }
       if (*abort) return;
-      const int w = w_b - i / a.n_slices, slice = i % a.n_slices;
       const int rows = min(TOK, a.L - slice * TOK);
       const uint32_t bytes = (uint32_t)rows * D * 2;
       const size_t off = ((size_t)bh * a.N + a.S + (size_t)w * a.L + (size_t)slice * TOK) * D;
@@ -487,6 +490,8 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
       ptx::mbar_expect_tx(bar, 2 * bytes);
       bulk_load(dst, a.K + off, bytes, bar);
       bulk_load(dst + kSliceBytes, a.V + off, bytes, bar);
+      if (++kr[g] == ring) { kr[g] = 0; ++use[g]; }
+      if (++slice == a.n_slices) { slice = 0; --w; }
     }
     return;
   }
@@ -497,6 +502,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
   const float inv_dof = 1.0f / (float)(D - a.ddof);
   const uint32_t PINF = 0x7F807F80u, NINF = 0xFF80FF80u;
   uint32_t st[2][2][4];  // running [K,V][min,max][4 bf16 pairs] of this group's slices of the window
+  int it_all = 0, ckr = 0, cuse = 0;   // slices streamed so far by both groups; this group's ring position
   for (int wi = 0; wi < n_win; ++wi) {
    const int w = w_b - wi;
    const bool scoring = wi > 0;          // the first window streamed is a reference only
@@ -524,14 +530,13 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
    }
 #pragma unroll
    for (int j = 0; j < 4; ++j) { st[0][0][j] = st[1][0][j] = PINF; st[0][1][j] = st[1][1][j] = NINF; }
-   for (int i = wi * a.n_slices; i < (wi + 1) * a.n_slices; ++i) {
-    if (i % kChainGroups != grp) continue;
-    const int slice = i % a.n_slices;
-    const int k = i / kChainGroups, slot = grp * ring + k % ring;
+   for (int slice = 0; slice < a.n_slices; ++slice, ++it_all) {
+    if ((it_all & 1) != grp) continue;
+    const int slot = grp * ring + ckr;   // this group's slice number k: ckr = k % ring, cuse = k / ring
     // One barrier per slice: a warp whose wait ran out skips the arithmetic (warp-uniform, the
     // arithmetic shuffles), raises the flag and still meets the group at the barrier below, after
     // which every thread of the group reads the same verdict.
-    bool got = stage_wait(ptx::smem_u32(&full_bar[slot]), (k / ring) & 1, a.spin_limit);
+    bool got = stage_wait(ptx::smem_u32(&full_bar[slot]), cuse & 1, a.spin_limit);
     got = __all_sync(0xffffffffu, got);
     if (!got) {
       *abort = 1;
@@ -638,6 +643,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
     group_sync(grp);   // every read of the stage by this group is done
     if (*abort) break;   // written before the barrier by whichever thread gave up
     if (gt == 0) ptx::mbar_arrive(ptx::smem_u32(&empty_bar[slot]));
+    if (++ckr == ring) { ckr = 0; ++cuse; }
    }
 
    // ---- end of window w: both groups have written their spreads and hold their part of the statistics ----
