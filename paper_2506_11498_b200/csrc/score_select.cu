@@ -471,9 +471,9 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
       if (use[g] > 0 && !stage_wait(ptx::smem_u32(&empty_bar[slot]), (use[g] - 1) & 1, a.spin_limit)) {
         *abort = 1;
         atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT);
-        return;
+        break;
       }
-      if (*abort) return;
+      if (*abort) break;
       const int rows = min(TOK, a.L - slice * TOK);
       const uint32_t bytes = (uint32_t)rows * D * 2;
       const size_t off = ((size_t)bh * a.N + a.S + (size_t)w * a.L + (size_t)slice * TOK) * D;
@@ -485,7 +485,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
           ((reinterpret_cast<uintptr_t>(a.K + off) | reinterpret_cast<uintptr_t>(a.V + off) | dst) & 15u)) {
         *abort = 1;
         atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT);
-        return;
+        break;
       }
       ptx::mbar_expect_tx(bar, 2 * bytes);
       bulk_load(dst, a.K + off, bytes, bar);
@@ -493,6 +493,13 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
       if (++kr[g] == ring) { kr[g] = 0; ++use[g]; }
       if (++slice == a.n_slices) { slice = 0; --w; }
     }
+    // No copy may be in flight when the CTA's shared memory is released, whether the run completed or a
+    // wait gave up: the producer leaves last, after the latest copy into every slot has landed (bounded).
+    for (int g = 0; g < kChainGroups; ++g)
+      for (int r = 0; r < ring; ++r) {
+        const int u = r < kr[g] ? use[g] : use[g] - 1;   // latest use of the slot that was issued
+        if (u >= 0) (void)stage_wait(ptx::smem_u32(&full_bar[g * ring + r]), u & 1, a.spin_limit);
+      }
     return;
   }
 
