@@ -305,32 +305,42 @@ lrsa_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
   if (tid == 0 && abort_s) atomicExch(a.status, (int)LRSA_ERR_TIMEOUT);
 }
 
-// Per query row: D~_t = sum_c dO[t,c] * O[t,c] and -LSE_t * log2(e), one warp per row.
+// Per query row: D~_t = sum_c dO[t,c] * O[t,c] and -LSE_t * log2(e).  d/8 lanes share a row (16 bytes
+// each) and a warp takes kPrepUnroll groups of 256/d rows with all loads issued before the arithmetic:
+// the kernel only streams O and dO once and should run at memory speed.
+constexpr int kPrepUnroll = 4;
 __global__ void bwd_prep_kernel(const __nv_bfloat16* __restrict__ O, const __nv_bfloat16* __restrict__ dO,
                                 const float* __restrict__ LSE, float2* __restrict__ stats, long long rows, int d) {
-  const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (row >= rows) return;
   const int lane = threadIdx.x & 31;
-  float acc = 0.f;
-  if ((d & 127) == 0) {   // 8 bytes per lane and load: a 128-element row in one load per tensor
-    for (int c = lane * 4; c < d; c += 128) {
-      const uint2 o = *reinterpret_cast<const uint2*>(O + row * d + c);
-      const uint2 g = *reinterpret_cast<const uint2*>(dO + row * d + c);
-      acc = fmaf(__uint_as_float(o.x << 16), __uint_as_float(g.x << 16), acc);
-      acc = fmaf(__uint_as_float(o.x & 0xffff0000u), __uint_as_float(g.x & 0xffff0000u), acc);
-      acc = fmaf(__uint_as_float(o.y << 16), __uint_as_float(g.y << 16), acc);
-      acc = fmaf(__uint_as_float(o.y & 0xffff0000u), __uint_as_float(g.y & 0xffff0000u), acc);
-    }
-  } else {
-    for (int c = lane * 2; c < d; c += 64) {
-      const __nv_bfloat162 o = *reinterpret_cast<const __nv_bfloat162*>(O + row * d + c);
-      const __nv_bfloat162 g = *reinterpret_cast<const __nv_bfloat162*>(dO + row * d + c);
-      acc += __bfloat162float(o.x) * __bfloat162float(g.x) + __bfloat162float(o.y) * __bfloat162float(g.y);
+  const int lpr = d >> 3, rpw = 32 / lpr;   // lanes per row, rows per warp-wide load (d = 64: 8, 4; d = 128: 16, 2)
+  const long long warp_id = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long row0 = warp_id * (kPrepUnroll * rpw) + lane / lpr;
+  const int c = (lane % lpr) * 8;
+  uint4 o[kPrepUnroll], g[kPrepUnroll];
+#pragma unroll
+  for (int u = 0; u < kPrepUnroll; ++u) {
+    const long long row = row0 + u * rpw;
+    if (row < rows) {
+      o[u] = *reinterpret_cast<const uint4*>(O + row * d + c);
+      g[u] = *reinterpret_cast<const uint4*>(dO + row * d + c);
+    } else {
+      o[u] = make_uint4(0, 0, 0, 0);
+      g[u] = make_uint4(0, 0, 0, 0);
     }
   }
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-  if (lane == 0) stats[row] = make_float2(-LSE[row] * 1.4426950408889634f, acc);
+  for (int u = 0; u < kPrepUnroll; ++u) {
+    const uint32_t ow[4] = {o[u].x, o[u].y, o[u].z, o[u].w}, gw[4] = {g[u].x, g[u].y, g[u].z, g[u].w};
+    float acc = 0.f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      acc = fmaf(__uint_as_float(ow[j] << 16), __uint_as_float(gw[j] << 16), acc);
+      acc = fmaf(__uint_as_float(ow[j] & 0xffff0000u), __uint_as_float(gw[j] & 0xffff0000u), acc);
+    }
+    for (int off = lpr >> 1; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    const long long row = row0 + u * rpw;
+    if ((lane % lpr) == 0 && row < rows) stats[row] = make_float2(-LSE[row] * 1.4426950408889634f, acc);
+  }
 }
 
 // kbar[bh][c] += (1/N) * sum of K[bh][t][c] over this block's rows (kbar zeroed beforehand).
@@ -369,7 +379,8 @@ __global__ void __launch_bounds__(256) kbar_kernel(const __nv_bfloat16* __restri
 int launch_bwd_prep(const Geom& g, const __nv_bfloat16* O, const __nv_bfloat16* dO, const float* LSE,
                     const __nv_bfloat16* K, float2* stats, float* kbar, cudaStream_t st) {
   const long long rows = (long long)g.B * g.Hq * g.N;
-  bwd_prep_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(O, dO, LSE, stats, rows, g.d);
+  const long long rows_per_block = 8LL * kPrepUnroll * (32 / (g.d >> 3));
+  bwd_prep_kernel<<<(unsigned)((rows + rows_per_block - 1) / rows_per_block), 256, 0, st>>>(O, dO, LSE, stats, rows, g.d);
   LRSA_CUDA_CHECK(cudaGetLastError());
   launch_counter().n++;
   const int nsplit = 64, rpb = (g.N + nsplit - 1) / nsplit;
