@@ -285,30 +285,43 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     red_s[half][row] = l;
     asm volatile("bar.sync 1, 256;" ::: "memory");   // the eight softmax warps, whether or not a wait gave up
     if (ok) ok = mbar_wait(smem_u32(&bars.pv_done), (n - 1) & 1, abort);
+    // The output rows go through shared memory (the Q tile and the first ring slot are idle by now) and
+    // leave as one bulk copy per row: per-thread 16-byte stores to rows 256 bytes apart cost a
+    // transaction each.  Rows are padded by 16 bytes so that a warp's stores spread over the banks.
+    constexpr int kRowBytes = D * 2, kStageStride = kRowBytes + 16;
+    unsigned char* stage_out = smem_raw + (sQ - smem_u32(smem_raw));
+    const bool store = qpos < rb.q_end;
     if (ok) {
       tc_fence_after_sync();
       const float lt = red_s[0][row] + red_s[1][row];
       const float inv = 1.0f / lt;
-      const bool store = qpos < rb.q_end;
-      __nv_bfloat16* orow = a.O + ((size_t)bh * a.N + qpos) * D + half * (D / 2);
+      unsigned char* srow = stage_out + row * kStageStride + half * (kRowBytes / 2);
 #pragma unroll
       for (int q = 0; q < D / 64; ++q) {
         uint32_t o[32];
         tmem_ld32(O_addr + q * 32, o);
         tmem_wait_ld();
-        if (store) {
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            uint4 w;
-            w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
-            w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
-            w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
-            w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-            *reinterpret_cast<uint4*>(orow + q * 32 + v * 8) = w;
-          }
+        for (int v = 0; v < 4; ++v) {
+          uint4 w;
+          w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+          w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+          w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+          w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+          *reinterpret_cast<uint4*>(srow + (q * 4 + v) * 16) = w;
         }
       }
       if (store && half == 0) a.LSE[(size_t)bh * a.N + qpos] = m * a.scale + logf(lt);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the bulk copy reads these stores
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");   // both halves of every row are staged (or a wait gave up)
+    if (half == 0 && store && !*abort) {
+      __nv_bfloat16* orow = a.O + ((size_t)bh * a.N + qpos) * D;
+      asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(orow),
+                   "r"(smem_u32(stage_out + row * kStageStride)), "r"((uint32_t)kRowBytes)
+                   : "memory");
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory is released at exit
     }
   }
 
