@@ -185,7 +185,7 @@ def run_reference(args, w):
 
 
 # DRAM bytes per backward call (dK/dV + dQ kernels) from the ncu summary under profiles/, per workload
-BWD_DRAM_BYTES = {"cfg2_32k_gqa7_d128": 3.085e9}
+BWD_DRAM_BYTES = {"cfg2_32k_gqa7_d128": 3.075e9}
 
 
 def main():

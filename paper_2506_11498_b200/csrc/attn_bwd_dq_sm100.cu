@@ -270,32 +270,45 @@ lrsa_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
     red_s[half][row] = rsum;
     asm volatile("bar.sync 1, 256;" ::: "memory");   // the eight softmax warps, whether or not a wait gave up
     if (ok) ok = mbar_wait(smem_u32(&bars.acc_done), 0, abort);
+    // The dQ rows go through shared memory (the Q and dO tiles are idle since their copy into tensor
+    // memory) and leave as one bulk copy per row: per-thread 16-byte stores to rows 256 bytes apart cost
+    // a transaction each.  Rows are padded by 16 bytes so that a warp's stores spread over the banks.
+    constexpr int kRowBytes = D * 2, kStageStride = kRowBytes + 16;
+    unsigned char* stage_out = smem_raw + (sQ - smem_u32(smem_raw));
     if (ok) {
       tc_fence_after_sync();
       const float r = red_s[0][row] + red_s[1][row];
       constexpr int CH = D / 2;   // output columns of this warpgroup
       const uint32_t A_addr = tmem + lane_addr + Cfg::kColA + half * CH;
       const float* kb = a.kbar + (size_t)bh_kv * D + half * CH;
-      __nv_bfloat16* orow = a.dQ + ((size_t)bh * a.N + qpos) * D + half * CH;
+      unsigned char* srow = stage_out + row * kStageStride + half * (kRowBytes / 2);
 #pragma unroll
       for (int q = 0; q < CH / 32; ++q) {
         uint32_t o[32];
         tmem_ld32(A_addr + q * 32, o);
         tmem_wait_ld();
-        if (live) {
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            float f[8];
+        for (int v = 0; v < 4; ++v) {
+          float f[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e)
-              f[e] = fmaf(-r, __ldg(kb + q * 32 + 8 * v + e), __uint_as_float(o[8 * v + e])) * a.scale;
-            uint4 w;
-            w.x = pack_bf16(f[0], f[1]); w.y = pack_bf16(f[2], f[3]);
-            w.z = pack_bf16(f[4], f[5]); w.w = pack_bf16(f[6], f[7]);
-            *reinterpret_cast<uint4*>(orow + q * 32 + v * 8) = w;
-          }
+          for (int e = 0; e < 8; ++e)
+            f[e] = fmaf(-r, __ldg(kb + q * 32 + 8 * v + e), __uint_as_float(o[8 * v + e])) * a.scale;
+          uint4 w;
+          w.x = pack_bf16(f[0], f[1]); w.y = pack_bf16(f[2], f[3]);
+          w.z = pack_bf16(f[4], f[5]); w.w = pack_bf16(f[6], f[7]);
+          *reinterpret_cast<uint4*>(srow + (q * 4 + v) * 16) = w;
         }
       }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the bulk copy reads these stores
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");   // both halves of every row are staged (or a wait gave up)
+    if (half == 0 && live && !*abort) {
+      __nv_bfloat16* orow = a.dQ + ((size_t)bh * a.N + qpos) * D;
+      asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(orow),
+                   "r"(smem_u32(stage_out + row * kStageStride)), "r"((uint32_t)kRowBytes)
+                   : "memory");
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory is released at exit
     }
   }
 
