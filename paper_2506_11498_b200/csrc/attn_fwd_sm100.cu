@@ -58,6 +58,7 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) FwdBars bars;
   __shared__ float red_s[2][kTile];   // [column half][row] partial row sums
+  __shared__ unsigned short loaded_s[2][kTile];   // [column half][row] tiles whose S this softmax thread has read
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
 
@@ -84,6 +85,7 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     }
     fence_barrier_init();
   }
+  if (tid < 2 * kTile) (&loaded_s[0][0])[tid] = 0;
   if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_s), 512); tmem_relinquish(); }
   tc_fence_before_sync();
   __syncthreads();
@@ -200,6 +202,8 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     tc_fence_before_sync();
     mbar_arrive(smem_u32(&bars.qt_ready));   // also when the wait gave up: the issuers then see abort
     float m = -INFINITY, l = 0.f;
+    volatile unsigned short* my_loaded = &loaded_s[half][row];
+    volatile unsigned short* partner_loaded = &loaded_s[1 - half][row];
     for (int j = 0; j < n && ok; ++j) {
       const int b = j & 1;
       ok = mbar_wait(smem_u32(&bars.s_full[b]), (j >> 1) & 1, abort);
@@ -213,6 +217,7 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       tmem_ld32(S_oth, *reinterpret_cast<uint32_t(*)[32]>(&t[0]));
       tmem_ld32(S_oth + 32, *reinterpret_cast<uint32_t(*)[32]>(&t[32]));
       tmem_wait_ld();
+      *my_loaded = (unsigned short)(j + 1);   // the partner may now overwrite its S columns of this tile with P
       // keys of the tile this row may see: the first `limit`
       const int limit = j < n_ct ? rb.n_front - j * kTile : qpos - (rb.dense_start + (j - n_ct) * kTile) + 1;
       if (limit < kTile) {
@@ -277,6 +282,18 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       }
       f2_unpack(sum2, sum0, sum1);
       l += sum0 + sum1;
+      // The two threads of a row read each other's S columns above and overwrite their own with P below:
+      // a thread stores only after its partner has published that it has loaded this tile.  By now the
+      // partner has had a whole tile of arithmetic to do so, so the check practically never waits.
+      if ((int)*partner_loaded <= j) {
+        const long long t0 = clock64();
+        while ((int)*partner_loaded <= j) {
+          if (*abort) { ok = false; break; }
+          if (clock64() - t0 > kWaitCycles) { *abort = 1; ok = false; break; }
+        }
+      }
+      ok = __all_sync(0xffffffffu, ok);   // one verdict per warp: the store below is warp-wide
+      if (!ok) break;
       tmem_st32(S_own, pk);   // over the first half of this warpgroup's own S columns
       tmem_wait_st();
       tc_fence_before_sync();
@@ -424,6 +441,7 @@ static int launch_fwd_t(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat
   a.status = status;
   const long long grid = (long long)a.plan.total * a.BH;
   if (grid > 0x7fffffffLL) return LRSA_ERR_UNSUPPORTED;
+  if (g.N / kTile + 4 > 0xffff) return LRSA_ERR_UNSUPPORTED;   // 16-bit tile counters of the softmax threads
   auto kern = lrsa_fwd_kernel<D>;
   LRSA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem));
   kern<<<(unsigned)grid, Cfg::kThreads, Cfg::kSmem, st>>>(mQ, mK, mV, mKc, mVc, a);

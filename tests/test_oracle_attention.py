@@ -125,6 +125,31 @@ def test_hand_enumerated_mask():
         assert (orc.visible_row(p, idx, 0, 0, t) == rows[t]).all(), t
 
 
+def test_hand_enumerated_mask_previous_window_compressed():
+    """The n_dense_prev = 0 variant against masks enumerated by hand (two cases: every window
+    followed by a full one, and a tail that leaves the last window uncompressed)."""
+    cases, cur = [], None
+    for line in open(os.path.join(GOLD, "mask_ndp0_worked_example.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        k, *v = line.split()
+        if k == "case":
+            cur = {"N": int(v[2]), "S": int(v[4]), "L": int(v[6]), "K": int(v[8]), "rows": {}}
+            cases.append(cur)
+        elif k == "kept":
+            cur["kept"] = [int(x) for x in v]
+        else:
+            cur["rows"][int(k)] = np.array([c == "1" for c in v[0]])
+    assert len(cases) == 2
+    for c in cases:
+        p = orc.OracleParams(1, 1, 1, c["N"], 2, c["L"], c["K"], c["S"], n_dense_prev=0)
+        wsel = orc.geometry(p)["Wsel"]
+        idx = np.array(c["kept"], np.int32).reshape(1, 1, wsel, c["K"])
+        assert len(c["rows"]) == c["N"]
+        for t in range(c["N"]):
+            assert (orc.visible_row(p, idx, 0, 0, t) == c["rows"][t]).all(), (c["N"], t)
+
+
 def test_full_retention_is_dense_causal():
     """K = L keeps everything: results equal textbook causal attention for any idx."""
     B, Hq, Hkv, N, d, L, S = 1, 4, 2, 70, 16, 16, 3
