@@ -1,8 +1,9 @@
 // LRSA attention backward, dK / dV part, on tcgen05 tensor cores (key-outer).
 //
 // The keys of one (batch, KV head) are cut into 128-row tiles of two kinds:
-//   compact tiles : rows of the compact sinks+kept buffer; seen by every query of the chunks that
-//                   see those windows compressed
+//   compact tiles : 128 consecutive entries of the sinks + kept-positions list (the condensed KV cache
+//                   of Section 3.2, gathered from K and V by position when the CTA starts); seen by
+//                   every query of the chunks that see those windows compressed
 //   dense tiles   : original positions of one window (or of the sink region / the tail); seen
 //                   causally by the queries from the diagonal to the end of the last chunk that
 //                   still sees that window uncompressed
@@ -20,9 +21,9 @@
 // afterwards) needs.  The list of a tile runs from the last query tile backwards with the heads
 // innermost, and compact tiles are launched segment by segment, so that the CTAs resident at one time
 // read the same Q_i / dO_i tiles (L2 hits instead of one DRAM pass per key tile).  At the end
-// the accumulators are added (fp32 atomics) to a zeroed workspace indexed by original position
-// (dense tiles) or by compact row (compact tiles); two small kernels then fold the compact rows
-// onto their original positions and convert to bf16.
+// the accumulators are added (fp32 atomics) to a zeroed workspace indexed by original position: a
+// row of a compact tile goes to the position it was gathered from, so a kept key's compressed and
+// uncompressed contributions meet in one row.  A small kernel then converts to bf16.
 #include "attn_common_sm100.h"
 
 namespace lrsa {
@@ -180,12 +181,13 @@ struct DkvCfg {
 struct DkvArgs {
   DkvPlan plan;
   int BHkv, Hq, Hkv, total_segs;
+  const int32_t* idx;    // [B*Hkv][n_kept] kept positions, ascending
+  int n_kept;            // Wsel * K
   const float2* stats;   // per query row: (-LSE * log2(e), D~ = rowsum(dO * O) from the bf16 O)
   float* Dacc;           // [B*Hq][N], zeroed: receives sum_j P_tj dP_tj, the accurate D for the dQ kernel
   const int2* seg_map;   // launch order: (tile, segment of the tile)
-  float* dKf;   // [BHkv][N + Rc][D] fp32, zeroed
+  float* dKf;   // [BHkv][N][D] fp32, zeroed
   float* dVf;
-  int rows_ws;  // N + Rc
   float scale, scale_log2;
   int* status;
 };
@@ -204,7 +206,7 @@ template <int D>
 __global__ void __launch_bounds__(DkvCfg<D>::kThreads, 1)
 lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapdO,
                     const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
-                    const __grid_constant__ CUtensorMap mapKc, const __grid_constant__ CUtensorMap mapVc,
+                    const __grid_constant__ CUtensorMap mapKg, const __grid_constant__ CUtensorMap mapVg,
                     const DkvArgs a) {
   using Cfg = DkvCfg<D>;
   constexpr int NS = Cfg::kStages;
@@ -256,12 +258,23 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     // ---------------- producer (whole warp: lanes stage LSE and D, lane 0 drives TMA) ----------------
     if (lane == 0) {
       prefetch_tensormap(&mapQ); prefetch_tensormap(&mapdO);
-      const CUtensorMap* mk = kt.kind == 0 ? &mapKc : &mapK;
-      const CUtensorMap* mv = kt.kind == 0 ? &mapVc : &mapV;
       mbar_expect_tx(smem_u32(&bars.kv_full), 2 * Cfg::kKTileBytes);
+    }
+    __syncwarp();
+    if (kt.kind == 0) {
+      // every lane gathers four rows of the list tile from their positions in K and V
+      const int32_t* kept = a.idx + (size_t)bh_kv * a.n_kept;
+      int pos[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) pos[i] = bh_kv * p.N + compact_row_pos(kept, p.S, p.Rc, kt.row0 + 4 * lane + i);
       for (int h = 0; h < Cfg::kSub; ++h) {
-        tma_load_3d(sK + h * Cfg::kKSubBytes, mk, h * 64, kt.row0, bh_kv, smem_u32(&bars.kv_full));
-        tma_load_3d(sV + h * Cfg::kKSubBytes, mv, h * 64, kt.row0, bh_kv, smem_u32(&bars.kv_full));
+        tma_gather4_2d(sK + h * Cfg::kKSubBytes + lane * 512, &mapKg, h * 64, pos[0], pos[1], pos[2], pos[3], smem_u32(&bars.kv_full));
+        tma_gather4_2d(sV + h * Cfg::kKSubBytes + lane * 512, &mapVg, h * 64, pos[0], pos[1], pos[2], pos[3], smem_u32(&bars.kv_full));
+      }
+    } else if (lane == 0) {
+      for (int h = 0; h < Cfg::kSub; ++h) {
+        tma_load_3d(sK + h * Cfg::kKSubBytes, &mapK, h * 64, kt.row0, bh_kv, smem_u32(&bars.kv_full));
+        tma_load_3d(sV + h * Cfg::kKSubBytes, &mapV, h * 64, kt.row0, bh_kv, smem_u32(&bars.kv_full));
       }
     }
     bool ok = true;
@@ -516,8 +529,11 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
       // warpgroup 0 adds dK (scaled), warpgroup 1 adds dV
       const uint32_t acc = tmem + lane_addr + (wg == 0 ? Cfg::kColK : Cfg::kColV);
       const float mul = wg == 0 ? a.scale : 1.0f;
-      const int out_row = kt.kind == 0 ? p.N + kt.row0 + r : kt.row0 + r;
-      float* dst = (wg == 0 ? a.dKf : a.dVf) + ((size_t)bh_kv * a.rows_ws + out_row) * D;
+      // a row of a compact tile lands on the position it was gathered from
+      const int out_row = kt.kind == 0
+                              ? compact_row_pos(a.idx + (size_t)bh_kv * a.n_kept, p.S, p.Rc, kt.row0 + r)
+                              : kt.row0 + r;
+      float* dst = (wg == 0 ? a.dKf : a.dVf) + ((size_t)bh_kv * p.N + out_row) * D;
 #pragma unroll
       for (int q = 0; q < D / 32; ++q) {
         uint32_t o[32];
@@ -539,30 +555,14 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
   if (tid == 0 && abort_s) atomicExch(a.status, (int)LRSA_ERR_TIMEOUT);
 }
 
-// dense[pos(r)] += compact[r] for every compact row (positions are distinct), one warp per row
-__global__ void fold_compact_kernel(float* dKf, float* dVf, const int32_t* __restrict__ idx, int BHkv, int N, int Rc,
-                                    int S, int n_kept, int d) {
-  const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (wid >= (long long)BHkv * Rc) return;
-  const int bh = (int)(wid / Rc), r = (int)(wid % Rc), lane = threadIdx.x & 31;
-  const int pos = r < S ? r : idx[(size_t)bh * n_kept + (r - S)];
-  const size_t base = (size_t)bh * (N + Rc);
-  for (int c = lane; c < d; c += 32) {
-    dKf[(base + pos) * d + c] += dKf[(base + N + r) * d + c];
-    dVf[(base + pos) * d + c] += dVf[(base + N + r) * d + c];
-  }
-}
-
-// bf16 outputs from the fp32 accumulation rows [0, N) of every (batch, KV head)
+// bf16 outputs from the fp32 accumulators [BHkv][N][d]; n4 = number of float4 groups
 __global__ void convert_dkv_kernel(const float* __restrict__ dKf, const float* __restrict__ dVf,
-                                   __nv_bfloat16* __restrict__ dK, __nv_bfloat16* __restrict__ dV, long long n4,
-                                   long long row_elems_out, long long row_elems_ws) {
-  // n4 = number of float4 groups over [BHkv][N][d]; row_elems_* = N*d and (N+Rc)*d
+                                   __nv_bfloat16* __restrict__ dK, __nv_bfloat16* __restrict__ dV, long long n4) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n4) return;
-  const long long e = i * 4, bh = e / row_elems_out, off = e % row_elems_out;
-  const float4 k = *reinterpret_cast<const float4*>(dKf + bh * row_elems_ws + off);
-  const float4 v = *reinterpret_cast<const float4*>(dVf + bh * row_elems_ws + off);
+  const long long e = i * 4;
+  const float4 k = *reinterpret_cast<const float4*>(dKf + e);
+  const float4 v = *reinterpret_cast<const float4*>(dVf + e);
   uint2 ko, vo;
   ko.x = pack_bf16(k.x, k.y); ko.y = pack_bf16(k.z, k.w);
   vo.x = pack_bf16(v.x, v.y); vo.y = pack_bf16(v.z, v.w);
@@ -584,7 +584,7 @@ size_t dkv_ws_bytes(const Geom& g, size_t* prefix_bytes) {
   const size_t cnt = align_up((size_t)(p.n_tiles + 1) * sizeof(int), 1024);
   const size_t pre = cnt + align_up((size_t)(dkv_total_segs(p) + 1) * sizeof(int2), 1024);
   if (prefix_bytes) *prefix_bytes = pre;
-  const size_t acc = align_up((size_t)g.B * g.Hkv * (g.N + g.Rc) * g.d * sizeof(float), 1024);
+  const size_t acc = align_up((size_t)g.B * g.Hkv * g.N * g.d * sizeof(float), 1024);
   return pre + 2 * acc;
 }
 
@@ -602,10 +602,10 @@ static int launch_dkv_t(const Geom& g, const DkvArgs& a, const CUtensorMap* m, c
   return LRSA_OK;
 }
 
-// ws_dkv: region of dkv_ws_bytes(g) bytes.  Zeroes the accumulators, runs the tile kernel, folds the
-// compact rows onto their positions and writes bf16 dK, dV.
+// ws_dkv: region of dkv_ws_bytes(g) bytes.  Zeroes the accumulators, runs the tile kernel and writes
+// bf16 dK, dV.
 int launch_bwd_dkv_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO, const __nv_bfloat16* K,
-                         const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, const float2* stats,
+                         const __nv_bfloat16* V, const float2* stats,
                          float* Dacc, const int32_t* idx, __nv_bfloat16* dK, __nv_bfloat16* dV, void* ws_dkv,
                          int* status, cudaStream_t st) {
   const DkvPlan p = make_dkv_plan(g);
@@ -625,30 +625,22 @@ int launch_bwd_dkv_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloa
   const int total_segs = dkv_total_segs(p);
 
   CUtensorMap m[6];
-  const long long rc = g.Rc > 0 ? g.Rc : 1;
   int r = make_tmap_bf16(&m[0], Q, g.d, g.N, (long long)g.B * g.Hq, kQRows);
   if (r == LRSA_OK) r = make_tmap_bf16(&m[1], dO, g.d, g.N, (long long)g.B * g.Hq, kQRows);
   if (r == LRSA_OK) r = make_tmap_bf16(&m[2], K, g.d, g.N, (long long)g.B * g.Hkv, kTile);
   if (r == LRSA_OK) r = make_tmap_bf16(&m[3], V, g.d, g.N, (long long)g.B * g.Hkv, kTile);
-  if (r == LRSA_OK) r = make_tmap_bf16(&m[4], Kc, g.d, rc, (long long)g.B * g.Hkv, kTile);
-  if (r == LRSA_OK) r = make_tmap_bf16(&m[5], Vc, g.d, rc, (long long)g.B * g.Hkv, kTile);
+  if (r == LRSA_OK) r = make_tmap_bf16_rows(&m[4], K, g.d, (long long)g.B * g.Hkv * g.N);
+  if (r == LRSA_OK) r = make_tmap_bf16_rows(&m[5], V, g.d, (long long)g.B * g.Hkv * g.N);
   if (r != LRSA_OK) return r;
   DkvArgs a;
   a.plan = p; a.BHkv = g.B * g.Hkv; a.Hq = g.Hq; a.Hkv = g.Hkv; a.total_segs = total_segs;
-  a.stats = stats; a.Dacc = Dacc; a.seg_map = seg_map; a.dKf = dKf; a.dVf = dVf; a.rows_ws = g.N + g.Rc;
+  a.idx = idx; a.n_kept = g.Wsel * g.K;
+  a.stats = stats; a.Dacc = Dacc; a.seg_map = seg_map; a.dKf = dKf; a.dVf = dVf;
   a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f; a.status = status;
   r = g.d == 128 ? launch_dkv_t<128>(g, a, m, st) : launch_dkv_t<64>(g, a, m, st);
   if (r != LRSA_OK) return r;
-  if (g.Rc > 0) {
-    const long long warps = (long long)a.BHkv * g.Rc;
-    fold_compact_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(dKf, dVf, idx, a.BHkv, g.N, g.Rc, g.S,
-                                                                    g.Wsel * g.K, g.d);
-    LRSA_CUDA_CHECK(cudaGetLastError());
-    launch_counter().n++;
-  }
   const long long n4 = (long long)a.BHkv * g.N * g.d / 4;
-  convert_dkv_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(dKf, dVf, dK, dV, n4, (long long)g.N * g.d,
-                                                                  (long long)(g.N + g.Rc) * g.d);
+  convert_dkv_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(dKf, dVf, dK, dV, n4);
   LRSA_CUDA_CHECK(cudaGetLastError());
   launch_counter().n++;
   return LRSA_OK;

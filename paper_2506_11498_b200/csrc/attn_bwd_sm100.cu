@@ -5,7 +5,7 @@ namespace lrsa {
 namespace {
 
 struct BwdWs {
-  size_t kbar, dacc, kc, vc, stats, dkv, total;
+  size_t kbar, dacc, zero_end, kc, vc, stats, dkv, total;
 };
 BwdWs bwd_ws_layout(const Geom& g) {
   BwdWs w;
@@ -15,7 +15,8 @@ BwdWs bwd_ws_layout(const Geom& g) {
   // cleared together with the header: the mean-key accumulator and the per-row D accumulator
   w.kbar = off; off += align_up((size_t)g.B * g.Hkv * g.d * sizeof(float), 1024);
   w.dacc = off; off += align_up((size_t)g.B * g.Hq * g.N * sizeof(float), 1024);
-  w.kc = off; off += cbytes;
+  w.zero_end = off;
+  w.kc = off; off += cbytes;   // compact K/V for the query-outer dQ kernel
   w.vc = off; off += cbytes;
   w.stats = off; off += align_up((size_t)g.B * g.Hq * g.N * sizeof(float2), 1024);
   w.dkv = off; off += dkv_ws_bytes(g, nullptr);
@@ -33,7 +34,7 @@ int launch_attn_bwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bflo
                           __nv_bfloat16* dV, void* ws, cudaStream_t st) {
   const BwdWs lay = bwd_ws_layout(g);
   unsigned char* base = static_cast<unsigned char*>(ws);
-  LRSA_CUDA_CHECK(cudaMemsetAsync(base, 0, lay.kc, st));
+  LRSA_CUDA_CHECK(cudaMemsetAsync(base, 0, lay.zero_end, st));
   launch_counter().n++;
   __nv_bfloat16* Kc = reinterpret_cast<__nv_bfloat16*>(base + lay.kc);
   __nv_bfloat16* Vc = reinterpret_cast<__nv_bfloat16*>(base + lay.vc);
@@ -41,10 +42,9 @@ int launch_attn_bwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bflo
   float* kbar = reinterpret_cast<float*>(base + lay.kbar);
   float* Dacc = reinterpret_cast<float*>(base + lay.dacc);
   int* status = &reinterpret_cast<WsHeader*>(base)->status;
-  int rc = launch_compact_kv(g, K, V, idx, Kc, Vc, st);
-  if (rc == LRSA_OK) rc = launch_bwd_prep(g, O, dO, LSE, K, stats, kbar, st);
-  if (rc == LRSA_OK)
-    rc = launch_bwd_dkv_sm100(g, Q, dO, K, V, Kc, Vc, stats, Dacc, idx, dK, dV, base + lay.dkv, status, st);
+  int rc = launch_bwd_prep(g, O, dO, LSE, K, stats, kbar, st);
+  if (rc == LRSA_OK) rc = launch_bwd_dkv_sm100(g, Q, dO, K, V, stats, Dacc, idx, dK, dV, base + lay.dkv, status, st);
+  if (rc == LRSA_OK) rc = launch_compact_kv(g, K, V, idx, Kc, Vc, st);
   if (rc == LRSA_OK) rc = launch_bwd_dq_sm100(g, Q, dO, K, V, Kc, Vc, stats, Dacc, kbar, dQ, status, st);
   return rc;
 }

@@ -95,8 +95,23 @@ __device__ __forceinline__ RowBlock decode_block(const BlockPlan& p, int blk) {
 int make_tmap_bf16(CUtensorMap* map, const void* base, int d, long long rows, long long outer, int box_rows);
 
 // Gathers the sink rows and the kept rows of K and V into the compact buffers
-// Kc, Vc [B*Hkv][Rc][d] (the condensed KV cache of Section 3.2).
+// Kc, Vc [B*Hkv][Rc][d] (the condensed KV cache of Section 3.2) for the query-outer kernels, which
+// stream the list once per query tile: a TMA row gather in their main loops was measured at about
+// 6 bytes per clock and SM, a fifth of what they consume.
 int launch_compact_kv(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat16* V, const int32_t* idx,
                       __nv_bfloat16* Kc, __nv_bfloat16* Vc, cudaStream_t st);
+
+// 2-D bf16 tensor map over [rows][d] with a (64 x 1) box and 128-byte swizzle, for row gathers
+// (tile::gather4).  The key-outer dK/dV kernel loads its one list tile per CTA this way, four rows per
+// copy, straight from K and V into the swizzled operand tile.
+int make_tmap_bf16_rows(CUtensorMap* map, const void* base, int d, long long rows);
+
+// Original position of row r of the compact (sinks + kept) key list of one (batch, KV head); `kept`
+// points at that head's idx entries.  Rows at or beyond n_rows are never used by a product (their scores
+// are masked); they map to position 0 so that the row fetched for them is valid, finite data.
+__device__ __forceinline__ int compact_row_pos(const int32_t* __restrict__ kept, int S, int n_rows, int r) {
+  if (r >= n_rows) return 0;
+  return r < S ? r : __ldg(kept + (r - S));
+}
 
 }  // namespace lrsa

@@ -408,6 +408,19 @@ int make_tmap_bf16(CUtensorMap* map, const void* base, int d, long long rows, lo
   return r == CUDA_SUCCESS ? LRSA_OK : LRSA_ERR_CUDA;
 }
 
+int make_tmap_bf16_rows(CUtensorMap* map, const void* base, int d, long long rows) {
+  EncodeFn fn = encode_fn();
+  if (!fn) return LRSA_ERR_CUDA;
+  cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+  cuuint32_t box[2] = {64, 1};
+  cuuint32_t es[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? LRSA_OK : LRSA_ERR_CUDA;
+}
+
 int launch_compact_kv(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat16* V, const int32_t* idx,
                       __nv_bfloat16* Kc, __nv_bfloat16* Vc, cudaStream_t st) {
   if (g.Rc == 0) return LRSA_OK;

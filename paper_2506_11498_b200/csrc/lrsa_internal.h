@@ -97,7 +97,7 @@ int launch_bwd_dq_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat
 
 size_t dkv_ws_bytes(const Geom& g, size_t* prefix_bytes);
 int launch_bwd_dkv_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO, const __nv_bfloat16* K,
-                         const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, const float2* stats,
+                         const __nv_bfloat16* V, const float2* stats,
                          float* Dacc, const int32_t* idx, __nv_bfloat16* dK, __nv_bfloat16* dV, void* ws_dkv,
                          int* status, cudaStream_t st);
 

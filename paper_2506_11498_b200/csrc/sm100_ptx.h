@@ -1,6 +1,6 @@
 // Thin inline-PTX wrappers for the Blackwell (sm_100a) features the attention kernels use:
-// mbarriers, TMA tile loads, tensor memory (TMEM) management and tcgen05 MMA.
-// Every wait is bounded by the caller (see mbar_wait in attn_sm100.cu).
+// mbarriers, TMA tile and row-gather loads, tensor memory (TMEM) management and tcgen05 MMA.
+// Every wait is bounded by the caller (see mbar_wait in attn_common_sm100.h).
 #pragma once
 
 #include <cuda.h>
@@ -67,6 +67,16 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+// ---- TMA: four rows of a 2-D tensor (box = 64 elements x 1 row) gathered into four consecutive
+// 128-byte rows of shared memory; c0 is the element column (a multiple of 8 for bf16), r0..r3 the rows ----
+__device__ __forceinline__ void tma_gather4_2d(uint32_t dst, const CUtensorMap* map, int c0, int r0, int r1, int r2,
+                                               int r3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
       : "memory");
 }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
