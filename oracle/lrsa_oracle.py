@@ -194,3 +194,127 @@ def attn_bwd(p, Q, K, V, dO, idx):
     dQ = bwd_rows(p, Q, K, V, dO, idx, all_rows(p)).reshape(p.B, p.Hq, p.N, p.d)
     dK, dV = bwd_keys(p, Q, K, V, dO, idx, all_keys(p))
     return dQ, dK.reshape(p.B, p.Hkv, p.N, p.d), dV.reshape(p.B, p.Hkv, p.N, p.d)
+
+
+# ----------------------------------------------------------------------------------------------
+# Packed variable-length batches.  Several sequences lie back to back along the token axis of every
+# [B, H, N, d] tensor; `cu` (length n_seqs + 1, cu[0] = 0, cu[-1] = N) holds their boundaries.  Each
+# sequence is an independent LRSA problem with its own sinks and lag windows counted from its own first
+# token (Section 3.2 describes one sequence; nothing crosses a boundary), so every function below is
+# the single-sequence function applied to each slice, with positions shifted by the slice's start.
+# Scored windows are numbered sequence after sequence; kept positions are positions in the packed axis.
+# ----------------------------------------------------------------------------------------------
+
+def _seq(p: OracleParams, n: int) -> OracleParams:
+    from dataclasses import replace
+    return replace(p, N=int(n))
+
+
+def _slice(a: np.ndarray, lo: int, hi: int) -> np.ndarray:
+    return np.ascontiguousarray(a[:, :, lo:hi])
+
+
+def packed_windows(p: OracleParams, cu) -> list:
+    """Per sequence: (first token, length, scored windows, index of its first scored window)."""
+    out, woff = [], 0
+    for s in range(len(cu) - 1):
+        n = int(cu[s + 1] - cu[s])
+        wsel = geometry(_seq(p, n))["Wsel"]
+        out.append((int(cu[s]), n, wsel, woff))
+        woff += wsel
+    return out
+
+
+def score_select_packed(p: OracleParams, K: np.ndarray, V: np.ndarray, cu):
+    seqs = packed_windows(p, cu)
+    total = sum(s[2] for s in seqs)
+    idx = np.zeros((p.B, p.Hkv, total, p.K), np.int32)
+    sc = np.zeros((p.B, p.Hkv, total, p.L), np.float64)
+    for t0, n, wsel, woff in seqs:
+        if wsel == 0:
+            continue
+        i, s = score_select(_seq(p, n), _slice(K, t0, t0 + n), _slice(V, t0, t0 + n))
+        idx[:, :, woff:woff + wsel] = i + t0
+        sc[:, :, woff:woff + wsel] = s
+    return idx, sc
+
+
+def _local_idx(idx: np.ndarray, t0: int, wsel: int, woff: int) -> np.ndarray:
+    return np.ascontiguousarray(idx[:, :, woff:woff + wsel] - t0).astype(np.int32)
+
+
+def visible_row_packed(p: OracleParams, idx: np.ndarray, cu, b: int, hkv: int, t: int) -> np.ndarray:
+    out = np.zeros(int(cu[-1]), bool)
+    for t0, n, wsel, woff in packed_windows(p, cu):
+        if t0 <= t < t0 + n:
+            out[t0:t0 + n] = visible_row(_seq(p, n), _local_idx(idx, t0, wsel, woff), b, hkv, t - t0)
+    return out
+
+
+def attn_fwd_packed(p, Q, K, V, idx, cu):
+    O = np.zeros((p.B, p.Hq, int(cu[-1]), p.d), np.float64)
+    LSE = np.zeros((p.B, p.Hq, int(cu[-1])), np.float64)
+    for t0, n, wsel, woff in packed_windows(p, cu):
+        o, l = attn_fwd(_seq(p, n), _slice(Q, t0, t0 + n), _slice(K, t0, t0 + n), _slice(V, t0, t0 + n),
+                        _local_idx(idx, t0, wsel, woff))
+        O[:, :, t0:t0 + n] = o
+        LSE[:, :, t0:t0 + n] = l
+    return O, LSE
+
+
+def attn_bwd_packed(p, Q, K, V, dO, idx, cu):
+    N = int(cu[-1])
+    dQ = np.zeros((p.B, p.Hq, N, p.d), np.float64)
+    dK = np.zeros((p.B, p.Hkv, N, p.d), np.float64)
+    dV = np.zeros((p.B, p.Hkv, N, p.d), np.float64)
+    for t0, n, wsel, woff in packed_windows(p, cu):
+        q, k, v = attn_bwd(_seq(p, n), _slice(Q, t0, t0 + n), _slice(K, t0, t0 + n), _slice(V, t0, t0 + n),
+                           _slice(dO, t0, t0 + n), _local_idx(idx, t0, wsel, woff))
+        dQ[:, :, t0:t0 + n] = q
+        dK[:, :, t0:t0 + n] = k
+        dV[:, :, t0:t0 + n] = v
+    return dQ, dK, dV
+
+
+def _by_sequence(p, cu, rows):
+    """Groups (b, h, t) triples by the sequence that holds t: yields (sequence, positions in `rows`)."""
+    rows = np.asarray(rows, np.int32)
+    for seq in packed_windows(p, cu):
+        sel = np.flatnonzero((rows[:, 2] >= seq[0]) & (rows[:, 2] < seq[0] + seq[1]))
+        if sel.size:
+            yield seq, sel
+
+
+def fwd_rows_packed(p, Q, K, V, idx, cu, rows):
+    rows = np.asarray(rows, np.int32)
+    O = np.zeros((len(rows), p.d), np.float64)
+    LSE = np.zeros(len(rows), np.float64)
+    for (t0, n, wsel, woff), sel in _by_sequence(p, cu, rows):
+        loc = rows[sel].copy()
+        loc[:, 2] -= t0
+        O[sel], LSE[sel] = fwd_rows(_seq(p, n), _slice(Q, t0, t0 + n), _slice(K, t0, t0 + n), _slice(V, t0, t0 + n),
+                                    _local_idx(idx, t0, wsel, woff), loc)
+    return O, LSE
+
+
+def bwd_rows_packed(p, Q, K, V, dO, idx, cu, rows):
+    rows = np.asarray(rows, np.int32)
+    dQ = np.zeros((len(rows), p.d), np.float64)
+    for (t0, n, wsel, woff), sel in _by_sequence(p, cu, rows):
+        loc = rows[sel].copy()
+        loc[:, 2] -= t0
+        dQ[sel] = bwd_rows(_seq(p, n), _slice(Q, t0, t0 + n), _slice(K, t0, t0 + n), _slice(V, t0, t0 + n),
+                           _slice(dO, t0, t0 + n), _local_idx(idx, t0, wsel, woff), loc)
+    return dQ
+
+
+def bwd_keys_packed(p, Q, K, V, dO, idx, cu, keys):
+    keys = np.asarray(keys, np.int32)
+    dK = np.zeros((len(keys), p.d), np.float64)
+    dV = np.zeros((len(keys), p.d), np.float64)
+    for (t0, n, wsel, woff), sel in _by_sequence(p, cu, keys):
+        loc = keys[sel].copy()
+        loc[:, 2] -= t0
+        dK[sel], dV[sel] = bwd_keys(_seq(p, n), _slice(Q, t0, t0 + n), _slice(K, t0, t0 + n), _slice(V, t0, t0 + n),
+                                    _slice(dO, t0, t0 + n), _local_idx(idx, t0, wsel, woff), loc)
+    return dK, dV
