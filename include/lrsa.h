@@ -19,6 +19,12 @@
  * Geometry : positions [0, S) are sinks.  Window w covers [S + w*L, S + (w+1)*L).
  *            W = floor((N-S)/L) full windows, tail T = N - S - W*L (< L) tokens.
  *            W_sel = max(W-1, 0) windows have a full following window and are scored.
+ * Packed   : with n_seqs > 0 each sequence [cu_seqlens[s], cu_seqlens[s+1]) is an independent problem
+ *            (Section 3.2 applied to it alone): its sinks and windows are counted from its first token
+ *            (a sequence shorter than S is all sinks) and no query sees another sequence.  Scored
+ *            windows are numbered sequence after sequence, W_sel is their total, and kept positions
+ *            are positions on the packed token axis.  The sequences are processed one after the
+ *            other on the stream.
  * Stream   : `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
  *            enqueue work and return without synchronising.  Two calls that use the same
  *            workspace must be ordered (same stream, or otherwise serialised).
@@ -42,7 +48,7 @@ extern "C" {
 typedef enum lrsa_status {
   LRSA_OK = 0,
   LRSA_ERR_INVALID_ARG = 1,         /* null pointer, non-positive size, K > L, Hq % Hkv != 0, misaligned */
-  LRSA_ERR_UNSUPPORTED = 2,         /* head_dim not in {64,128}, chunk != lag, seq_len < n_sink, ... */
+  LRSA_ERR_UNSUPPORTED = 2,         /* head_dim not in {64,128}, chunk not a multiple of lag, seq_len < n_sink, ... */
   LRSA_ERR_WORKSPACE_TOO_SMALL = 3,
   LRSA_ERR_CUDA = 4,                /* CUDA runtime error while enqueueing */
   LRSA_ERR_TIMEOUT = 5              /* a bounded device-side wait expired */
@@ -54,7 +60,9 @@ typedef struct lrsa_params {
   int32_t n_kv_heads;    /* Hkv */
   int32_t seq_len;       /* N >= n_sink */
   int32_t head_dim;      /* d in {64, 128} */
-  int32_t chunk;         /* query chunk size; must equal lag */
+  int32_t chunk;         /* query chunk size: a positive multiple of lag.  The mask of Section 3.2 does not
+                            depend on how many lag windows are filled at a time ("the number of filling chunks
+                            can be optimized"), so every multiple gives the results of chunk == lag */
   int32_t lag;           /* L, lag window size */
   int32_t top_k;         /* K = r*L kept tokens per window, 1 <= K <= L */
   int32_t n_sink;        /* S >= 0 */
@@ -62,6 +70,10 @@ typedef struct lrsa_params {
                             paper's "sliding window"); 0: it is compressed too when scored */
   int32_t std_ddof;      /* divisor of the per-token Std is head_dim - std_ddof; 0 or 1 */
   float softmax_scale;   /* 0 -> 1/sqrt(head_dim) as in Eq. 3 */
+  int32_t n_seqs;        /* 0: every batch element is one sequence of seq_len tokens.  > 0: packed batch, the
+                            token axis of every batch element holds n_seqs sequences back to back */
+  const int32_t* cu_seqlens; /* HOST pointer, n_seqs + 1 boundaries: cu_seqlens[0] = 0, increasing,
+                            cu_seqlens[n_seqs] = seq_len.  Read during the call only.  NULL when n_seqs = 0 */
 } lrsa_params_t;
 
 /* Number of scored windows W_sel (see Geometry).  idx has W_sel * top_k entries per KV head. */
@@ -97,7 +109,8 @@ int lrsa_score_select(const lrsa_params_t* params, const void* K, const void* V,
  *
  *   - Allocates nothing: no cudaMalloc/cudaFree, no allocating library routine.  The caller still
  *     passes K, V (in) and idx, score (out; score may be NULL) exactly as for lrsa_score_select.
- *   - Problems whose scratch need (the score_select figure of lrsa_workspace_bytes) exceeds
+ *   - Problems whose scratch need (the score_select figure of lrsa_workspace_bytes: 256 bytes for lag
+ *     windows of up to 4096 tokens, counters, statistics and per-token spreads beyond) exceeds
  *     LRSA_STATIC_SCRATCH_BYTES are refused with LRSA_ERR_WORKSPACE_TOO_SMALL and nothing is
  *     enqueued; use lrsa_score_select with a workspace for those.
  *   - The device that owns `cuda_stream` must be the current device.  The first call on each device
@@ -111,6 +124,14 @@ int lrsa_score_select(const lrsa_params_t* params, const void* K, const void* V,
 #define LRSA_STATIC_SCRATCH_BYTES (4u << 20)
 int lrsa_score_select_static(const lrsa_params_t* params, const void* K, const void* V, int32_t* idx,
                              float* score, void* cuda_stream);
+
+/*
+ * What lrsa_workspace_status is for the calls that take a workspace: reads the status word that the last
+ * lrsa_score_select_static call on the current device left in the library's fixed array (the caller has
+ * no pointer to it).  Synchronises `cuda_stream`, allocates nothing.  Returns LRSA_OK, LRSA_ERR_TIMEOUT
+ * (a bounded device-side wait expired: idx and score are undefined), or LRSA_ERR_CUDA.
+ */
+int lrsa_score_select_static_status(void* cuda_stream);
 
 /*
  * LRSA attention forward (Section 3.1, Eq. 3 with the chunked mask of Section 3.2).

@@ -181,8 +181,9 @@ struct DkvCfg {
 struct DkvArgs {
   DkvPlan plan;
   int BHkv, Hq, Hkv, total_segs;
-  const int32_t* idx;    // [B*Hkv][n_kept] kept positions, ascending
-  int n_kept;            // Wsel * K
+  const int32_t* idx;    // kept positions of this sequence's windows: head bh at idx + bh * kept_stride
+  int kept_stride;       // Wtot * K entries per (batch, KV head)
+  int Nrow, tok0;        // tokens per (batch, head) row (the stride of every tensor); first token of the sequence
   const float2* stats;   // per query row: (-LSE * log2(e), D~ = rowsum(dO * O) from the bf16 O)
   float* Dacc;           // [B*Hq][N], zeroed: receives sum_j P_tj dP_tj, the accurate D for the dQ kernel
   const int2* seg_map;   // launch order: (tile, segment of the tile)
@@ -263,10 +264,11 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     __syncwarp();
     if (kt.kind == 0) {
       // every lane gathers four rows of the list tile from their positions in K and V
-      const int32_t* kept = a.idx + (size_t)bh_kv * a.n_kept;
+      const int32_t* kept = a.idx + (size_t)bh_kv * a.kept_stride;
       int pos[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) pos[i] = bh_kv * p.N + compact_row_pos(kept, p.S, p.Rc, kt.row0 + 4 * lane + i);
+      for (int i = 0; i < 4; ++i)
+        pos[i] = bh_kv * a.Nrow + compact_row_pos(kept, p.S, p.Rc, kt.row0 + 4 * lane + i, a.tok0);
       for (int h = 0; h < Cfg::kSub; ++h) {
         tma_gather4_2d(sK + h * Cfg::kKSubBytes + lane * 512, &mapKg, h * 64, pos[0], pos[1], pos[2], pos[3], smem_u32(&bars.kv_full));
         tma_gather4_2d(sV + h * Cfg::kKSubBytes + lane * 512, &mapVg, h * 64, pos[0], pos[1], pos[2], pos[3], smem_u32(&bars.kv_full));
@@ -288,7 +290,7 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 #pragma unroll
       for (int k = 0; k < kQRows / 32; ++k) {
         const int q = q0 + lane + 32 * k;
-        v[k] = q < kt.qend ? __ldg(a.stats + (size_t)hq * p.N + q) : make_float2(-INFINITY, 0.f);
+        v[k] = q < kt.qend ? __ldg(a.stats + (size_t)hq * a.Nrow + q) : make_float2(-INFINITY, 0.f);
       }
     };
     float2 cur[kQRows / 32], nxt[kQRows / 32];
@@ -520,7 +522,7 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         }
         const int col = 16 * ((lane >> 4) & 1) + 8 * ((lane >> 3) & 1) + 2 * (lane & 3) + ((lane >> 2) & 1);
         const int q = q0 + wg * 32 + col;
-        if (q < kt.qend) atomicAdd(a.Dacc + (size_t)hq * p.N + q, c8[0]);
+        if (q < kt.qend) atomicAdd(a.Dacc + (size_t)hq * a.Nrow + q, c8[0]);
       }
     }
     if (ok) ok = mbar_wait(smem_u32(&bars.acc_done), 0, abort);
@@ -531,9 +533,9 @@ lrsa_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
       const float mul = wg == 0 ? a.scale : 1.0f;
       // a row of a compact tile lands on the position it was gathered from
       const int out_row = kt.kind == 0
-                              ? compact_row_pos(a.idx + (size_t)bh_kv * a.n_kept, p.S, p.Rc, kt.row0 + r)
+                              ? compact_row_pos(a.idx + (size_t)bh_kv * a.kept_stride, p.S, p.Rc, kt.row0 + r, a.tok0)
                               : kt.row0 + r;
-      float* dst = (wg == 0 ? a.dKf : a.dVf) + ((size_t)bh_kv * p.N + out_row) * D;
+      float* dst = (wg == 0 ? a.dKf : a.dVf) + ((size_t)bh_kv * a.Nrow + out_row) * D;
 #pragma unroll
       for (int q = 0; q < D / 32; ++q) {
         uint32_t o[32];
@@ -584,7 +586,7 @@ size_t dkv_ws_bytes(const Geom& g, size_t* prefix_bytes) {
   const size_t cnt = align_up((size_t)(p.n_tiles + 1) * sizeof(int), 1024);
   const size_t pre = cnt + align_up((size_t)(dkv_total_segs(p) + 1) * sizeof(int2), 1024);
   if (prefix_bytes) *prefix_bytes = pre;
-  const size_t acc = align_up((size_t)g.B * g.Hkv * g.N * g.d * sizeof(float), 1024);
+  const size_t acc = align_up((size_t)g.B * g.Hkv * g.Nrow * g.d * sizeof(float), 1024);
   return pre + 2 * acc;
 }
 
@@ -602,48 +604,70 @@ static int launch_dkv_t(const Geom& g, const DkvArgs& a, const CUtensorMap* m, c
   return LRSA_OK;
 }
 
-// ws_dkv: region of dkv_ws_bytes(g) bytes.  Zeroes the accumulators, runs the tile kernel and writes
-// bf16 dK, dV.
-int launch_bwd_dkv_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO, const __nv_bfloat16* K,
-                         const __nv_bfloat16* V, const float2* stats,
-                         float* Dacc, const int32_t* idx, __nv_bfloat16* dK, __nv_bfloat16* dV, void* ws_dkv,
-                         int* status, cudaStream_t st) {
-  const DkvPlan p = make_dkv_plan(g);
+// ws_dkv: region of dkv_ws_bytes(whole row) bytes.  Three steps: dkv_zero clears the fp32 accumulators of
+// the whole row, launch_bwd_dkv_sm100 runs the tile kernel of one sequence (its launch-order table is
+// rebuilt in the region's prefix, in stream order), dkv_convert writes bf16 dK, dV.
+static void dkv_regions(const Geom& whole, void* ws_dkv, int** seg_cnt, int2** seg_map, float** dKf, float** dVf,
+                        size_t* acc_bytes) {
   size_t pre = 0;
-  const size_t total = dkv_ws_bytes(g, &pre);
+  const size_t total = dkv_ws_bytes(whole, &pre);
   unsigned char* base = static_cast<unsigned char*>(ws_dkv);
-  const size_t acc = (total - pre) / 2;
-  int* seg_cnt = reinterpret_cast<int*>(base);
-  int2* seg_map = reinterpret_cast<int2*>(base + align_up((size_t)(p.n_tiles + 1) * sizeof(int), 1024));
-  float* dKf = reinterpret_cast<float*>(base + pre);
-  float* dVf = reinterpret_cast<float*>(base + pre + acc);
-  LRSA_CUDA_CHECK(cudaMemsetAsync(base + pre, 0, 2 * acc, st));
+  const DkvPlan p = make_dkv_plan(whole);
+  *acc_bytes = (total - pre) / 2;
+  *seg_cnt = reinterpret_cast<int*>(base);
+  *seg_map = reinterpret_cast<int2*>(base + align_up((size_t)(p.n_tiles + 1) * sizeof(int), 1024));
+  *dKf = reinterpret_cast<float*>(base + pre);
+  *dVf = reinterpret_cast<float*>(base + pre + *acc_bytes);
+}
+
+int dkv_zero(const Geom& whole, void* ws_dkv, cudaStream_t st) {
+  int* seg_cnt; int2* seg_map; float *dKf, *dVf; size_t acc;
+  dkv_regions(whole, ws_dkv, &seg_cnt, &seg_map, &dKf, &dVf, &acc);
+  LRSA_CUDA_CHECK(cudaMemsetAsync(dKf, 0, 2 * acc, st));
   launch_counter().n++;
+  return LRSA_OK;
+}
+
+int dkv_convert(const Geom& whole, void* ws_dkv, __nv_bfloat16* dK, __nv_bfloat16* dV, cudaStream_t st) {
+  int* seg_cnt; int2* seg_map; float *dKf, *dVf; size_t acc;
+  dkv_regions(whole, ws_dkv, &seg_cnt, &seg_map, &dKf, &dVf, &acc);
+  const long long n4 = (long long)whole.B * whole.Hkv * whole.Nrow * whole.d / 4;
+  convert_dkv_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(dKf, dVf, dK, dV, n4);
+  LRSA_CUDA_CHECK(cudaGetLastError());
+  launch_counter().n++;
+  return LRSA_OK;
+}
+
+// `whole`: the geometry of the whole row (workspace layout); `g`: the sequence to process.
+int launch_bwd_dkv_sm100(const Geom& whole, const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO,
+                         const __nv_bfloat16* K, const __nv_bfloat16* V, const float2* stats, float* Dacc,
+                         const int32_t* idx, void* ws_dkv, int* status, cudaStream_t st) {
+  const DkvPlan p = make_dkv_plan(g);
+  int* seg_cnt; int2* seg_map; float *dKf, *dVf; size_t acc;
+  dkv_regions(whole, ws_dkv, &seg_cnt, &seg_map, &dKf, &dVf, &acc);
+  // a part of a row never needs more than the whole row; checked all the same
+  if (p.n_tiles > make_dkv_plan(whole).n_tiles || dkv_total_segs(p) > dkv_total_segs(make_dkv_plan(whole)))
+    return LRSA_ERR_WORKSPACE_TOO_SMALL;
   dkv_setup_kernel<<<1, 256, 0, st>>>(p, seg_cnt, seg_map);
   LRSA_CUDA_CHECK(cudaGetLastError());
   launch_counter().n++;
   const int total_segs = dkv_total_segs(p);
 
   CUtensorMap m[6];
-  int r = make_tmap_bf16(&m[0], Q, g.d, g.N, (long long)g.B * g.Hq, kQRows);
-  if (r == LRSA_OK) r = make_tmap_bf16(&m[1], dO, g.d, g.N, (long long)g.B * g.Hq, kQRows);
-  if (r == LRSA_OK) r = make_tmap_bf16(&m[2], K, g.d, g.N, (long long)g.B * g.Hkv, kTile);
-  if (r == LRSA_OK) r = make_tmap_bf16(&m[3], V, g.d, g.N, (long long)g.B * g.Hkv, kTile);
-  if (r == LRSA_OK) r = make_tmap_bf16_rows(&m[4], K, g.d, (long long)g.B * g.Hkv * g.N);
-  if (r == LRSA_OK) r = make_tmap_bf16_rows(&m[5], V, g.d, (long long)g.B * g.Hkv * g.N);
+  const size_t sh = (size_t)g.tok0 * g.d;
+  int r = make_tmap_bf16(&m[0], Q + sh, g.d, g.N, (long long)g.B * g.Hq, kQRows, g.Nrow);
+  if (r == LRSA_OK) r = make_tmap_bf16(&m[1], dO + sh, g.d, g.N, (long long)g.B * g.Hq, kQRows, g.Nrow);
+  if (r == LRSA_OK) r = make_tmap_bf16(&m[2], K + sh, g.d, g.N, (long long)g.B * g.Hkv, kTile, g.Nrow);
+  if (r == LRSA_OK) r = make_tmap_bf16(&m[3], V + sh, g.d, g.N, (long long)g.B * g.Hkv, kTile, g.Nrow);
+  if (r == LRSA_OK) r = make_tmap_bf16_rows(&m[4], K + sh, g.d, (long long)g.B * g.Hkv * g.Nrow - g.tok0);
+  if (r == LRSA_OK) r = make_tmap_bf16_rows(&m[5], V + sh, g.d, (long long)g.B * g.Hkv * g.Nrow - g.tok0);
   if (r != LRSA_OK) return r;
   DkvArgs a;
   a.plan = p; a.BHkv = g.B * g.Hkv; a.Hq = g.Hq; a.Hkv = g.Hkv; a.total_segs = total_segs;
-  a.idx = idx; a.n_kept = g.Wsel * g.K;
-  a.stats = stats; a.Dacc = Dacc; a.seg_map = seg_map; a.dKf = dKf; a.dVf = dVf;
+  a.idx = idx + (size_t)g.woff * g.K; a.kept_stride = g.Wtot * g.K; a.Nrow = g.Nrow; a.tok0 = g.tok0;
+  a.stats = stats + g.tok0; a.Dacc = Dacc + g.tok0; a.seg_map = seg_map; a.dKf = dKf + sh; a.dVf = dVf + sh;
   a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f; a.status = status;
-  r = g.d == 128 ? launch_dkv_t<128>(g, a, m, st) : launch_dkv_t<64>(g, a, m, st);
-  if (r != LRSA_OK) return r;
-  const long long n4 = (long long)a.BHkv * g.N * g.d / 4;
-  convert_dkv_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(dKf, dVf, dK, dV, n4);
-  LRSA_CUDA_CHECK(cudaGetLastError());
-  launch_counter().n++;
-  return LRSA_OK;
+  return g.d == 128 ? launch_dkv_t<128>(g, a, m, st) : launch_dkv_t<64>(g, a, m, st);
 }
 
 }  // namespace lrsa

@@ -45,7 +45,7 @@ struct DqCfg {
 
 struct DqArgs {
   BlockPlan plan;
-  int BH, Hq, Hkv, G, N;
+  int BH, Hq, Hkv, G, N;   // N: tokens per (batch, head) row of stats, Dacc and dQ (the row stride)
   const float2* stats;   // per query row: (-LSE*log2e, D~); only the first component is used here
   const float* Dacc;     // per query row: D = sum_j P dP
   const float* kbar;     // [B*Hkv][D] mean key
@@ -410,17 +410,19 @@ static int launch_dq_t(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat1
   using Cfg = DqCfg<D>;
   CUtensorMap mQ, mdO, mK, mV, mKc, mVc;
   const long long rc = g.Rc > 0 ? g.Rc : 1;
-  int r = make_tmap_bf16(&mQ, Q, D, g.N, (long long)g.B * g.Hq, kTile);
-  if (r == LRSA_OK) r = make_tmap_bf16(&mdO, dO, D, g.N, (long long)g.B * g.Hq, kTile);
-  if (r == LRSA_OK) r = make_tmap_bf16(&mK, K, D, g.N, (long long)g.B * g.Hkv, kKeys);
-  if (r == LRSA_OK) r = make_tmap_bf16(&mV, V, D, g.N, (long long)g.B * g.Hkv, kKeys);
+  // the sequence starts at token tok0 of rows of Nrow tokens: shifted bases, rows beyond its end read as zero
+  const size_t sh = (size_t)g.tok0 * D;
+  int r = make_tmap_bf16(&mQ, Q + sh, D, g.N, (long long)g.B * g.Hq, kTile, g.Nrow);
+  if (r == LRSA_OK) r = make_tmap_bf16(&mdO, dO + sh, D, g.N, (long long)g.B * g.Hq, kTile, g.Nrow);
+  if (r == LRSA_OK) r = make_tmap_bf16(&mK, K + sh, D, g.N, (long long)g.B * g.Hkv, kKeys, g.Nrow);
+  if (r == LRSA_OK) r = make_tmap_bf16(&mV, V + sh, D, g.N, (long long)g.B * g.Hkv, kKeys, g.Nrow);
   if (r == LRSA_OK) r = make_tmap_bf16(&mKc, Kc, D, rc, (long long)g.B * g.Hkv, kKeys);
   if (r == LRSA_OK) r = make_tmap_bf16(&mVc, Vc, D, rc, (long long)g.B * g.Hkv, kKeys);
   if (r != LRSA_OK) return r;
   DqArgs a;
   a.plan = make_plan(g, kTile);
-  a.BH = g.B * g.Hq; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.N = g.N;
-  a.stats = stats; a.Dacc = Dacc; a.kbar = kbar; a.dQ = dQ;
+  a.BH = g.B * g.Hq; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.N = g.Nrow;
+  a.stats = stats + g.tok0; a.Dacc = Dacc + g.tok0; a.kbar = kbar; a.dQ = dQ + sh;
   a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f;
   a.status = status;
   const long long grid = (long long)a.plan.total * a.BH;

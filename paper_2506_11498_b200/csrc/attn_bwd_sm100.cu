@@ -28,7 +28,7 @@ BwdWs bwd_ws_layout(const Geom& g) {
 
 size_t attn_bwd_ws_bytes(const Geom& g) { return bwd_ws_layout(g).total; }
 
-int launch_attn_bwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
+int launch_attn_bwd_sm100(const lrsa_params_t* params, const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
                           const __nv_bfloat16* V, const __nv_bfloat16* O, const __nv_bfloat16* dO,
                           const float* LSE, const int32_t* idx, __nv_bfloat16* dQ, __nv_bfloat16* dK,
                           __nv_bfloat16* dV, void* ws, cudaStream_t st) {
@@ -42,10 +42,22 @@ int launch_attn_bwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bflo
   float* kbar = reinterpret_cast<float*>(base + lay.kbar);
   float* Dacc = reinterpret_cast<float*>(base + lay.dacc);
   int* status = &reinterpret_cast<WsHeader*>(base)->status;
+  // Per-row statistics and the mean key are taken over whole rows (the mean key is only a centring
+  // vector: any constant works).  Then, sequence after sequence, the dK/dV kernel (which also produces
+  // the accurate D of the sequence's rows) and the dQ kernel; bf16 dK, dV at the end.
   int rc = launch_bwd_prep(g, O, dO, LSE, K, stats, kbar, st);
-  if (rc == LRSA_OK) rc = launch_bwd_dkv_sm100(g, Q, dO, K, V, stats, Dacc, idx, dK, dV, base + lay.dkv, status, st);
-  if (rc == LRSA_OK) rc = launch_compact_kv(g, K, V, idx, Kc, Vc, st);
-  if (rc == LRSA_OK) rc = launch_bwd_dq_sm100(g, Q, dO, K, V, Kc, Vc, stats, Dacc, kbar, dQ, status, st);
+  if (rc == LRSA_OK) rc = dkv_zero(g, base + lay.dkv, st);
+  const int n_seqs = geom_n_seqs(params);
+  int woff = 0;
+  for (int s = 0; s < n_seqs && rc == LRSA_OK; ++s) {
+    Geom gs;
+    seq_geom(g, params->cu_seqlens, params->n_seqs, s, woff, &gs);
+    woff += gs.Wsel;
+    rc = launch_bwd_dkv_sm100(g, gs, Q, dO, K, V, stats, Dacc, idx, base + lay.dkv, status, st);
+    if (rc == LRSA_OK) rc = launch_compact_kv(gs, K, V, idx, Kc, Vc, st);
+    if (rc == LRSA_OK) rc = launch_bwd_dq_sm100(gs, Q, dO, K, V, Kc, Vc, stats, Dacc, kbar, dQ, status, st);
+  }
+  if (rc == LRSA_OK) rc = dkv_convert(g, base + lay.dkv, dK, dV, st);
   return rc;
 }
 

@@ -92,7 +92,10 @@ __device__ __forceinline__ RowBlock decode_block(const BlockPlan& p, int blk) {
 }
 
 // 3-D bf16 tensor map over [outer][rows][d] with a (64 x box_rows x 1) box and 128-byte swizzle.
-int make_tmap_bf16(CUtensorMap* map, const void* base, int d, long long rows, long long outer, int box_rows);
+// `row_stride`: rows between consecutive `outer` slices in memory (0: rows); larger when the map covers
+// one sequence of a packed row.
+int make_tmap_bf16(CUtensorMap* map, const void* base, int d, long long rows, long long outer, int box_rows,
+                   long long row_stride = 0);
 
 // Gathers the sink rows and the kept rows of K and V into the compact buffers
 // Kc, Vc [B*Hkv][Rc][d] (the condensed KV cache of Section 3.2) for the query-outer kernels, which
@@ -109,9 +112,10 @@ int make_tmap_bf16_rows(CUtensorMap* map, const void* base, int d, long long row
 // Original position of row r of the compact (sinks + kept) key list of one (batch, KV head); `kept`
 // points at that head's idx entries.  Rows at or beyond n_rows are never used by a product (their scores
 // are masked); they map to position 0 so that the row fetched for them is valid, finite data.
-__device__ __forceinline__ int compact_row_pos(const int32_t* __restrict__ kept, int S, int n_rows, int r) {
+// Positions are local to the sequence (kept entries are positions in the whole row, tok0 + local).
+__device__ __forceinline__ int compact_row_pos(const int32_t* __restrict__ kept, int S, int n_rows, int r, int tok0) {
   if (r >= n_rows) return 0;
-  return r < S ? r : __ldg(kept + (r - S));
+  return r < S ? r : __ldg(kept + (r - S)) - tok0;
 }
 
 }  // namespace lrsa

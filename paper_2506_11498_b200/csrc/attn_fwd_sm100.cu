@@ -35,7 +35,7 @@ struct FwdCfg {
 
 struct FwdArgs {
   BlockPlan plan;
-  int BH, Hq, Hkv, G, N;
+  int BH, Hq, Hkv, G, N;   // N: tokens per (batch, head) row of O and LSE (the row stride)
   __nv_bfloat16* O;
   float* LSE;
   float scale, scale_log2;   // softmax scale, and scale * log2(e)
@@ -348,15 +348,17 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   if (tid == 0 && abort_s) atomicExch(a.status, (int)LRSA_ERR_TIMEOUT);
 }
 
+// K, V point at the sequence's first token; `kept` entries are positions in the whole row (tok0 + local).
 __global__ void compact_kv_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
                                   const int32_t* __restrict__ idx, __nv_bfloat16* __restrict__ Kc,
-                                  __nv_bfloat16* __restrict__ Vc, int BHkv, int N, int d, int S, int n_kept, int Rc) {
+                                  __nv_bfloat16* __restrict__ Vc, int BHkv, int Nrow, int d, int S, int Rc, int tok0,
+                                  int kept_stride, int kept_off) {
   // one warp per compact row; a row is d*2 bytes = 8 (d=128) or 4 (d=64) bytes per lane
   const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (wid >= (long long)BHkv * Rc) return;
   const int bh = (int)(wid / Rc), r = (int)(wid % Rc), lane = threadIdx.x & 31;
-  const int pos = r < S ? r : idx[(size_t)bh * n_kept + (r - S)];
-  const size_t src = ((size_t)bh * N + pos) * d, dst = ((size_t)bh * Rc + r) * d;
+  const int pos = r < S ? r : idx[(size_t)bh * kept_stride + kept_off + (r - S)] - tok0;
+  const size_t src = ((size_t)bh * Nrow + pos) * d, dst = ((size_t)bh * Rc + r) * d;
   if (d == 128) {
     reinterpret_cast<uint2*>(Kc + dst)[lane] = reinterpret_cast<const uint2*>(K + src)[lane];
     reinterpret_cast<uint2*>(Vc + dst)[lane] = reinterpret_cast<const uint2*>(V + src)[lane];
@@ -395,11 +397,13 @@ FwdWs fwd_ws_layout(const Geom& g) {
 
 }  // namespace
 
-int make_tmap_bf16(CUtensorMap* map, const void* base, int d, long long rows, long long outer, int box_rows) {
+int make_tmap_bf16(CUtensorMap* map, const void* base, int d, long long rows, long long outer, int box_rows,
+                   long long row_stride) {
   EncodeFn fn = encode_fn();
   if (!fn) return LRSA_ERR_CUDA;
+  if (row_stride <= 0) row_stride = rows;
   cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)outer};
-  cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)d * 2 * (cuuint64_t)rows};
+  cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)d * 2 * (cuuint64_t)row_stride};
   cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
   cuuint32_t es[3] = {1, 1, 1};
   const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
@@ -426,7 +430,9 @@ int launch_compact_kv(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat16
   if (g.Rc == 0) return LRSA_OK;
   const long long warps = (long long)g.B * g.Hkv * g.Rc;
   const unsigned blocks = (unsigned)((warps + 7) / 8);
-  compact_kv_kernel<<<blocks, 256, 0, st>>>(K, V, idx, Kc, Vc, g.B * g.Hkv, g.N, g.d, g.S, g.Wsel * g.K, g.Rc);
+  const size_t sh = (size_t)g.tok0 * g.d;
+  compact_kv_kernel<<<blocks, 256, 0, st>>>(K + sh, V + sh, idx, Kc, Vc, g.B * g.Hkv, g.Nrow, g.d, g.S, g.Rc, g.tok0,
+                                            g.Wtot * g.K, g.woff * g.K);
   LRSA_CUDA_CHECK(cudaGetLastError());
   launch_counter().n++;
   return LRSA_OK;
@@ -441,16 +447,18 @@ static int launch_fwd_t(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat
   using Cfg = FwdCfg<D>;
   CUtensorMap mQ, mK, mV, mKc, mVc;
   const long long rc = g.Rc > 0 ? g.Rc : 1;
-  int rc_ = make_tmap_bf16(&mQ, Q, D, g.N, (long long)g.B * g.Hq, kTile);
-  if (rc_ == LRSA_OK) rc_ = make_tmap_bf16(&mK, K, D, g.N, (long long)g.B * g.Hkv, kTile);
-  if (rc_ == LRSA_OK) rc_ = make_tmap_bf16(&mV, V, D, g.N, (long long)g.B * g.Hkv, kTile);
+  // the sequence starts at token tok0 of rows of Nrow tokens: shifted bases, rows beyond its end read as zero
+  const size_t sh = (size_t)g.tok0 * D;
+  int rc_ = make_tmap_bf16(&mQ, Q + sh, D, g.N, (long long)g.B * g.Hq, kTile, g.Nrow);
+  if (rc_ == LRSA_OK) rc_ = make_tmap_bf16(&mK, K + sh, D, g.N, (long long)g.B * g.Hkv, kTile, g.Nrow);
+  if (rc_ == LRSA_OK) rc_ = make_tmap_bf16(&mV, V + sh, D, g.N, (long long)g.B * g.Hkv, kTile, g.Nrow);
   if (rc_ == LRSA_OK) rc_ = make_tmap_bf16(&mKc, Kc, D, rc, (long long)g.B * g.Hkv, kTile);
   if (rc_ == LRSA_OK) rc_ = make_tmap_bf16(&mVc, Vc, D, rc, (long long)g.B * g.Hkv, kTile);
   if (rc_ != LRSA_OK) return rc_;
   FwdArgs a;
   a.plan = make_plan(g, kTile);
-  a.BH = g.B * g.Hq; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.N = g.N;
-  a.O = O; a.LSE = LSE; a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f;
+  a.BH = g.B * g.Hq; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.N = g.Nrow;
+  a.O = O + sh; a.LSE = LSE + g.tok0; a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f;
   a.status = status;
   const long long grid = (long long)a.plan.total * a.BH;
   if (grid > 0x7fffffffLL) return LRSA_ERR_UNSUPPORTED;
@@ -463,19 +471,30 @@ static int launch_fwd_t(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat
   return LRSA_OK;
 }
 
-int launch_attn_fwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K, const __nv_bfloat16* V,
-                          const int32_t* idx, __nv_bfloat16* O, float* LSE, void* ws, cudaStream_t st) {
+int launch_attn_fwd_sm100(const lrsa_params_t* params, const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
+                          const __nv_bfloat16* V, const int32_t* idx, __nv_bfloat16* O, float* LSE, void* ws,
+                          cudaStream_t st) {
   const FwdWs lay = fwd_ws_layout(g);
   unsigned char* base = static_cast<unsigned char*>(ws);
   LRSA_CUDA_CHECK(cudaMemsetAsync(base, 0, sizeof(WsHeader), st));
   launch_counter().n++;
   __nv_bfloat16* Kc = reinterpret_cast<__nv_bfloat16*>(base + lay.kc);
   __nv_bfloat16* Vc = reinterpret_cast<__nv_bfloat16*>(base + lay.vc);
-  int rc = launch_compact_kv(g, K, V, idx, Kc, Vc, st);
-  if (rc != LRSA_OK) return rc;
   int* status = &reinterpret_cast<WsHeader*>(base)->status;
-  return g.d == 128 ? launch_fwd_t<128>(g, Q, K, V, Kc, Vc, O, LSE, status, st)
-                    : launch_fwd_t<64>(g, Q, K, V, Kc, Vc, O, LSE, status, st);
+  // sequence after sequence (one for an unpacked batch); the compact buffers are reused in stream order
+  const int n_seqs = geom_n_seqs(params);
+  int woff = 0;
+  for (int s = 0; s < n_seqs; ++s) {
+    Geom gs;
+    seq_geom(g, params->cu_seqlens, params->n_seqs, s, woff, &gs);
+    woff += gs.Wsel;
+    int rc = launch_compact_kv(gs, K, V, idx, Kc, Vc, st);
+    if (rc == LRSA_OK)
+      rc = gs.d == 128 ? launch_fwd_t<128>(gs, Q, K, V, Kc, Vc, O, LSE, status, st)
+                       : launch_fwd_t<64>(gs, Q, K, V, Kc, Vc, O, LSE, status, st);
+    if (rc != LRSA_OK) return rc;
+  }
+  return LRSA_OK;
 }
 
 }  // namespace lrsa

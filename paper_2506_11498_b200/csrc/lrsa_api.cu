@@ -23,7 +23,9 @@ int make_geom(const lrsa_params_t* p, Geom* g) {
   if (p->n_dense_prev != 0 && p->n_dense_prev != 1) return LRSA_ERR_INVALID_ARG;
   if (!(p->softmax_scale >= 0.f) || isinf(p->softmax_scale)) return LRSA_ERR_INVALID_ARG;
   if (p->head_dim != 64 && p->head_dim != 128) return LRSA_ERR_UNSUPPORTED;
-  if (p->chunk != p->lag) return LRSA_ERR_UNSUPPORTED;
+  // A query chunk of m lag windows sees exactly what m chunks of one window see (the mask of Section
+  // 3.2 does not depend on how many chunks are filled at a time), so any multiple of the lag is accepted.
+  if (p->chunk % p->lag != 0) return LRSA_ERR_UNSUPPORTED;
   if (p->seq_len < p->n_sink) return LRSA_ERR_UNSUPPORTED;
   if (p->lag > 32767) return LRSA_ERR_UNSUPPORTED;  // packed 16-bit counters in the selection scan
   if ((long long)p->batch * p->n_q_heads * p->seq_len > 0x7fffffffLL) return LRSA_ERR_UNSUPPORTED;
@@ -36,6 +38,52 @@ int make_geom(const lrsa_params_t* p, Geom* g) {
   g->C = g->W + (g->T > 0 ? 1 : 0);
   g->Wsel = g->W > 1 ? g->W - 1 : 0;
   g->Rc = g->S + g->Wsel * g->K;
+  g->Nrow = g->N; g->tok0 = 0; g->Wtot = g->Wsel; g->woff = 0;
+  if (p->n_seqs < 0) return LRSA_ERR_INVALID_ARG;
+  if (p->n_seqs > 0) {
+    if (!p->cu_seqlens || p->cu_seqlens[0] != 0 || p->cu_seqlens[p->n_seqs] != p->seq_len) return LRSA_ERR_INVALID_ARG;
+    int wtot = 0;
+    for (int s = 0; s < p->n_seqs; ++s) {
+      const int n = p->cu_seqlens[s + 1] - p->cu_seqlens[s];
+      if (n < 1) return LRSA_ERR_INVALID_ARG;
+      const int w = n > g->S ? (n - g->S) / g->L : 0;
+      wtot += w > 1 ? w - 1 : 0;
+    }
+    g->Wtot = wtot;
+  }
+  return LRSA_OK;
+}
+
+int geom_n_seqs(const lrsa_params_t* p) { return p->n_seqs > 0 ? p->n_seqs : 1; }
+
+void seq_geom(const Geom& whole, const int32_t* cu, int n_seqs, int s, int woff, Geom* out) {
+  *out = whole;
+  if (n_seqs <= 0 || !cu) return;   // the whole row is the one sequence
+  Geom& g = *out;
+  g.tok0 = cu[s];
+  g.N = cu[s + 1] - cu[s];
+  g.S = whole.S < g.N ? whole.S : g.N;   // a sequence shorter than the sink count is all sinks
+  g.W = (g.N - g.S) / g.L;
+  g.T = g.N - g.S - g.W * g.L;
+  g.C = g.W + (g.T > 0 ? 1 : 0);
+  g.Wsel = g.W > 1 ? g.W - 1 : 0;
+  g.Rc = g.S + g.Wsel * g.K;
+  g.woff = woff;
+}
+
+int run_score_select(const lrsa_params_t* p, const Geom& whole, const __nv_bfloat16* K, const __nv_bfloat16* V,
+                     int32_t* idx, float* score, void* ws, cudaStream_t st) {
+  LRSA_CUDA_CHECK(cudaMemsetAsync(ws, 0, sizeof(WsHeader), st));
+  launch_counter().n++;
+  const int n_seqs = geom_n_seqs(p);
+  int woff = 0;
+  for (int s = 0; s < n_seqs; ++s) {
+    Geom g;
+    seq_geom(whole, p->cu_seqlens, p->n_seqs, s, woff, &g);
+    const int rc = launch_score_select(g, K, V, idx, score, ws, st);
+    if (rc != LRSA_OK) return rc;
+    woff += g.Wsel;
+  }
   return LRSA_OK;
 }
 
@@ -61,7 +109,7 @@ int lrsa_num_sel_windows(const lrsa_params_t* params, int32_t* w_sel) {
   const int rc = make_geom(params, &g);
   if (rc != LRSA_OK) return rc;
   if (!w_sel) return LRSA_ERR_INVALID_ARG;
-  *w_sel = g.Wsel;
+  *w_sel = g.Wtot;
   return LRSA_OK;
 }
 
@@ -83,12 +131,12 @@ int lrsa_score_select(const lrsa_params_t* params, const void* K, const void* V,
   const int rc = make_geom(params, &g);
   if (rc != LRSA_OK) return rc;
   if (!K || !V || !workspace) return LRSA_ERR_INVALID_ARG;
-  if (g.Wsel > 0 && !idx) return LRSA_ERR_INVALID_ARG;
+  if (g.Wtot > 0 && !idx) return LRSA_ERR_INVALID_ARG;
   if (!aligned(K, 16) || !aligned(V, 16) || !aligned(idx, 4) || !aligned(score, 4) || !aligned(workspace, 256))
     return LRSA_ERR_INVALID_ARG;
   if (workspace_bytes < score_select_ws_bytes(g)) return LRSA_ERR_WORKSPACE_TOO_SMALL;
-  return launch_score_select(g, static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(V),
-                             idx, score, workspace, static_cast<cudaStream_t>(cuda_stream));
+  return run_score_select(params, g, static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(V),
+                          idx, score, workspace, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int lrsa_attn_fwd(const lrsa_params_t* params, const void* Q, const void* K, const void* V,
@@ -99,15 +147,16 @@ int lrsa_attn_fwd(const lrsa_params_t* params, const void* Q, const void* K, con
   const int rc = make_geom(params, &g);
   if (rc != LRSA_OK) return rc;
   if (!Q || !K || !V || !O || !LSE || !workspace) return LRSA_ERR_INVALID_ARG;
-  if (g.Wsel > 0 && !idx) return LRSA_ERR_INVALID_ARG;
+  if (g.Wtot > 0 && !idx) return LRSA_ERR_INVALID_ARG;
   if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(LSE, 16) ||
       !aligned(idx, 4) || !aligned(workspace, 256))
     return LRSA_ERR_INVALID_ARG;
   if (workspace_bytes < fwd_ws_bytes(g)) return LRSA_ERR_WORKSPACE_TOO_SMALL;
   auto st = static_cast<cudaStream_t>(cuda_stream);
-  auto fn = g_impl == 0 ? launch_attn_fwd_sm100 : launch_attn_ref_fwd;
-  return fn(g, static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K),
-            static_cast<const __nv_bfloat16*>(V), idx, static_cast<__nv_bfloat16*>(O), LSE, workspace, st);
+  auto bf = [](const void* p) { return static_cast<const __nv_bfloat16*>(p); };
+  if (g_impl == 0) return launch_attn_fwd_sm100(params, g, bf(Q), bf(K), bf(V), idx, static_cast<__nv_bfloat16*>(O), LSE, workspace, st);
+  if (params->n_seqs > 0) return LRSA_ERR_UNSUPPORTED;   // the validation kernels take one sequence per row
+  return launch_attn_ref_fwd(g, bf(Q), bf(K), bf(V), idx, static_cast<__nv_bfloat16*>(O), LSE, workspace, st);
 }
 
 int lrsa_attn_bwd(const lrsa_params_t* params, const void* Q, const void* K, const void* V,
@@ -118,7 +167,7 @@ int lrsa_attn_bwd(const lrsa_params_t* params, const void* Q, const void* K, con
   const int rc = make_geom(params, &g);
   if (rc != LRSA_OK) return rc;
   if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV || !workspace) return LRSA_ERR_INVALID_ARG;
-  if (g.Wsel > 0 && !idx) return LRSA_ERR_INVALID_ARG;
+  if (g.Wtot > 0 && !idx) return LRSA_ERR_INVALID_ARG;
   const void* ptrs[] = {Q, K, V, O, dO, LSE, dQ, dK, dV};
   for (const void* p : ptrs)
     if (!aligned(p, 16)) return LRSA_ERR_INVALID_ARG;
@@ -126,9 +175,12 @@ int lrsa_attn_bwd(const lrsa_params_t* params, const void* Q, const void* K, con
   if (workspace_bytes < bwd_ws_bytes(g)) return LRSA_ERR_WORKSPACE_TOO_SMALL;
   auto st = static_cast<cudaStream_t>(cuda_stream);
   auto bf = [](const void* p) { return static_cast<const __nv_bfloat16*>(p); };
-  auto fn = g_impl == 0 ? launch_attn_bwd_sm100 : launch_attn_ref_bwd;
-  return fn(g, bf(Q), bf(K), bf(V), bf(O), bf(dO), LSE, idx, static_cast<__nv_bfloat16*>(dQ),
-            static_cast<__nv_bfloat16*>(dK), static_cast<__nv_bfloat16*>(dV), workspace, st);
+  if (g_impl == 0)
+    return launch_attn_bwd_sm100(params, g, bf(Q), bf(K), bf(V), bf(O), bf(dO), LSE, idx, static_cast<__nv_bfloat16*>(dQ),
+                                 static_cast<__nv_bfloat16*>(dK), static_cast<__nv_bfloat16*>(dV), workspace, st);
+  if (params->n_seqs > 0) return LRSA_ERR_UNSUPPORTED;   // the validation kernels take one sequence per row
+  return launch_attn_ref_bwd(g, bf(Q), bf(K), bf(V), bf(O), bf(dO), LSE, idx, static_cast<__nv_bfloat16*>(dQ),
+                             static_cast<__nv_bfloat16*>(dK), static_cast<__nv_bfloat16*>(dV), workspace, st);
 }
 
 int lrsa_workspace_status(const void* workspace, void* cuda_stream) {

@@ -19,7 +19,18 @@ struct Geom {
   int C;     // query chunks = W + [T > 0]
   int Wsel;  // scored windows = max(W - 1, 0)
   int Rc;    // rows of the compact (sinks + kept) K/V buffer per KV head = S + Wsel*K
+  // Packed batches: this Geom describes ONE sequence of N tokens that starts at token `tok0` of rows
+  // that hold Nrow tokens per (batch, head); its scored windows are windows [woff, woff + Wsel) of the
+  // Wtot windows of the whole row.  Single sequence: Nrow = N, tok0 = 0, Wtot = Wsel, woff = 0.
+  // The launchers shift every tensor pointer by tok0 tokens and use Nrow as the row stride, so the
+  // kernels see an ordinary sequence; kept positions (idx) stay positions in the whole row.
+  int Nrow, tok0, Wtot, woff;
 };
+
+// Sequence s of a packed batch (cu = boundaries, n_seqs + 1 entries) as a Geom of its own.
+void seq_geom(const Geom& whole, const int32_t* cu, int n_seqs, int s, int woff, Geom* out);
+// Number of sequences and boundaries of `p` (a single sequence when it has no cu_seqlens).
+int geom_n_seqs(const lrsa_params_t* p);
 
 // Validates `p` and fills `g`. Returns an lrsa_status.
 int make_geom(const lrsa_params_t* p, Geom* g);
@@ -53,7 +64,11 @@ struct LaunchCounter {
 };
 LaunchCounter& launch_counter();
 
-// score_select.cu
+// lrsa_api.cu : clears the status header of `ws`, then scores and selects sequence after sequence.
+int run_score_select(const lrsa_params_t* p, const Geom& whole, const __nv_bfloat16* K, const __nv_bfloat16* V,
+                     int32_t* idx, float* score, void* ws, cudaStream_t st);
+
+// score_select.cu (one sequence; the status header of `ws` is cleared by the caller)
 size_t score_select_ws_bytes(const Geom& g);
 int launch_score_select(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat16* V, int32_t* idx,
                         float* score, void* ws, cudaStream_t st);
@@ -71,7 +86,7 @@ int launch_attn_ref_bwd(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat
 
 // attn_fwd_sm100.cu : tcgen05 / TMEM forward (workspace: header + compact K/V).
 size_t attn_fwd_ws_bytes(const Geom& g);
-int launch_attn_fwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
+int launch_attn_fwd_sm100(const lrsa_params_t* params, const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
                           const __nv_bfloat16* V, const int32_t* idx, __nv_bfloat16* O, float* LSE,
                           void* ws, cudaStream_t st);
 
@@ -82,7 +97,7 @@ int launch_attn_ref_bwd_dkv(const Geom& g, const __nv_bfloat16* Q, const __nv_bf
 
 // attn_bwd_*_sm100.cu : tcgen05 / TMEM backward.
 size_t attn_bwd_ws_bytes(const Geom& g);
-int launch_attn_bwd_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
+int launch_attn_bwd_sm100(const lrsa_params_t* params, const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K,
                           const __nv_bfloat16* V, const __nv_bfloat16* O, const __nv_bfloat16* dO,
                           const float* LSE, const int32_t* idx, __nv_bfloat16* dQ, __nv_bfloat16* dK,
                           __nv_bfloat16* dV, void* ws, cudaStream_t st);
@@ -96,10 +111,11 @@ int launch_bwd_dq_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat
                         const float* Dacc, const float* kbar, __nv_bfloat16* dQ, int* status, cudaStream_t st);
 
 size_t dkv_ws_bytes(const Geom& g, size_t* prefix_bytes);
-int launch_bwd_dkv_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO, const __nv_bfloat16* K,
-                         const __nv_bfloat16* V, const float2* stats,
-                         float* Dacc, const int32_t* idx, __nv_bfloat16* dK, __nv_bfloat16* dV, void* ws_dkv,
-                         int* status, cudaStream_t st);
+int dkv_zero(const Geom& whole, void* ws_dkv, cudaStream_t st);
+int launch_bwd_dkv_sm100(const Geom& whole, const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO,
+                         const __nv_bfloat16* K, const __nv_bfloat16* V, const float2* stats, float* Dacc,
+                         const int32_t* idx, void* ws_dkv, int* status, cudaStream_t st);
+int dkv_convert(const Geom& whole, void* ws_dkv, __nv_bfloat16* dK, __nv_bfloat16* dV, cudaStream_t st);
 
 #define LRSA_CUDA_CHECK(expr)                                 \
   do {                                                        \

@@ -15,6 +15,8 @@
 // A unit of window w waits only on units of window w+1, all of which hold smaller tickets, were
 // therefore picked up by CTAs that already run, and publish before they wait on anything: the
 // wait always ends, whatever the number of resident CTAs.  It is bounded all the same.
+#include <stddef.h>
+
 #include "lrsa_internal.h"
 #include "sm100_ptx.h"
 
@@ -34,7 +36,10 @@ struct ScoreArgs {
   int* done;      // [BH, Wsel]  slices of window w whose spreads are written
   uint32_t* mm;   // [BH, W, 2 (K,V), 2 (min,max), d] order-preserving keys, zero = identity
   float* spread;  // [BH, Wsel, 2 (K,V), L]
-  int BH, N, L, Kk, S, W, Wsel, n_slices, ddof;
+  int BH, N, L, Kk, S, W, Wsel, n_slices, ddof;   // N: tokens per (batch, head) row of K and V (the row stride)
+  int tok0, Wtot, woff;   // packed batches: K and V point at token tok0 of the rows; this sequence's windows are
+                          // [woff, woff + Wsel) of the Wtot windows per head of idx and score; positions are emitted + tok0
+  size_t elems;           // elements of K (and of V) from the shifted pointer to the end of the tensor
   int spin_limit;
 };
 
@@ -121,7 +126,7 @@ __device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* 
 #pragma unroll
   for (int i = 0; i < 8; ++i) { ek += red[i]; ev += red[8 + i]; }
   // Eq. 8
-  float* gs = a.score ? a.score + (size_t)(bh * a.Wsel + w) * L : nullptr;
+  float* gs = a.score ? a.score + (size_t)(bh * a.Wtot + a.woff + w) * L : nullptr;
   uint32_t kmin = 0xffffffffu, kmax = 0u;   // range of the keys (scores are positive: bit order = value order)
   for (int i = tid; i < L; i += kThreads) {
     const float s = sk[i] / ek + sv[i] / ev;
@@ -189,7 +194,8 @@ __device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* 
 
   // emit kept positions in ascending order: every thread takes a run of consecutive tokens, one block
   // scan gives the number of kept tokens before the run
-  int32_t* out = a.idx + (size_t)(bh * a.Wsel + w) * a.Kk;
+  int32_t* out = a.idx + (size_t)(bh * a.Wtot + a.woff + w) * a.Kk;
+  const int pos0 = a.tok0 + a.S + w * L;   // position of the window's first token in the row
   const int per = (L + kThreads - 1) / kThreads;
   const int i_lo = min(L, tid * per), i_hi = min(L, i_lo + per);
   int packed = 0;   // tokens above the K-th score | tokens equal to it << 16
@@ -214,10 +220,10 @@ __device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* 
   for (int i = i_lo; i < i_hi; ++i) {
     const uint32_t k = key[i];
     if (k > kth) {
-      out[gt_before + min(eq_before, need_eq)] = a.S + w * L + i;
+      out[gt_before + min(eq_before, need_eq)] = pos0 + i;
       ++gt_before;
     } else if (k == kth) {
-      if (eq_before < need_eq) out[gt_before + eq_before] = a.S + w * L + i;
+      if (eq_before < need_eq) out[gt_before + eq_before] = pos0 + i;
       ++eq_before;
     }
   }
@@ -481,7 +487,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
       const uint32_t dst = ptx::smem_u32(smem + slot * kStageBytes);
       // self-check: the slice lies inside the tensor and the copy is 16-byte granular; otherwise give up
       // (status word) instead of issuing it
-      if (w < 0 || w >= a.W || rows <= 0 || off + (size_t)rows * D > (size_t)a.BH * a.N * D || (bytes & 15u) ||
+      if (w < 0 || w >= a.W || rows <= 0 || off + (size_t)rows * D > a.elems || (bytes & 15u) ||
           ((reinterpret_cast<uintptr_t>(a.K + off) | reinterpret_cast<uintptr_t>(a.V + off) | dst) & 15u)) {
         *abort = 1;
         atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT);
@@ -724,24 +730,32 @@ ScoreWs score_ws_layout(const Geom& g) {
 
 }  // namespace
 
-size_t score_select_ws_bytes(const Geom& g) { return score_ws_layout(g).total; }
+// The chain kernel uses nothing but the status header; the one-slice-per-CTA kernel needs its counters,
+// statistics and spreads.
+size_t score_select_ws_bytes(const Geom& g) { return g.L <= kChainMaxL ? sizeof(WsHeader) : score_ws_layout(g).total; }
 
 int launch_score_select(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat16* V, int32_t* idx,
                         float* score, void* ws, cudaStream_t st) {
   if (g.Wsel == 0) return LRSA_OK;  // nothing is scored
   const ScoreWs lay = score_ws_layout(g);
   unsigned char* base = static_cast<unsigned char*>(ws);
-  // the chain kernel keeps everything but the status word on chip
-  LRSA_CUDA_CHECK(cudaMemsetAsync(base, 0, g.L <= kChainMaxL ? sizeof(WsHeader) : lay.zero_bytes, st));
-  launch_counter().n++;
+  // The status word (the header) is cleared once per call by the caller.  The chain kernel keeps everything
+  // else on chip; the one-slice-per-CTA kernel needs its ticket, counters and statistics at zero.
+  if (g.L > kChainMaxL) {
+    LRSA_CUDA_CHECK(cudaMemsetAsync(base + offsetof(WsHeader, ticket), 0, lay.zero_bytes - offsetof(WsHeader, ticket), st));
+    launch_counter().n++;
+  }
   ScoreArgs a;
-  a.K = K; a.V = V; a.idx = idx; a.score = score;
+  // the sequence starts at token tok0 of every row: shift the inputs, keep the row stride
+  a.K = K + (size_t)g.tok0 * g.d; a.V = V + (size_t)g.tok0 * g.d; a.idx = idx; a.score = score;
   a.hdr = reinterpret_cast<WsHeader*>(base);
   a.ready = reinterpret_cast<int*>(base + lay.ready);
   a.done = reinterpret_cast<int*>(base + lay.done);
   a.mm = reinterpret_cast<uint32_t*>(base + lay.mm);
   a.spread = reinterpret_cast<float*>(base + lay.spread);
-  a.BH = g.B * g.Hkv; a.N = g.N; a.L = g.L; a.Kk = g.K; a.S = g.S; a.W = g.W; a.Wsel = g.Wsel;
+  a.BH = g.B * g.Hkv; a.N = g.Nrow; a.L = g.L; a.Kk = g.K; a.S = g.S; a.W = g.W; a.Wsel = g.Wsel;
+  a.tok0 = g.tok0; a.Wtot = g.Wtot; a.woff = g.woff;
+  a.elems = ((size_t)g.B * g.Hkv * g.Nrow - (size_t)g.tok0) * g.d;
   a.ddof = g.ddof;
   a.spin_limit = 1 << 21;
   const int tok = g.d == 128 ? tok_per_unit<128>() : tok_per_unit<64>();

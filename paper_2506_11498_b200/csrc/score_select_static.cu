@@ -48,7 +48,7 @@ extern "C" int lrsa_score_select_static(const lrsa_params_t* params, const void*
   const int rc = make_geom(params, &g);
   if (rc != LRSA_OK) return rc;
   if (!K || !V) return LRSA_ERR_INVALID_ARG;
-  if (g.Wsel > 0 && !idx) return LRSA_ERR_INVALID_ARG;
+  if (g.Wtot > 0 && !idx) return LRSA_ERR_INVALID_ARG;
   auto misaligned = [](const void* p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a != 0; };
   if (misaligned(K, 16) || misaligned(V, 16) || misaligned(idx, 4) || misaligned(score, 4))
     return LRSA_ERR_INVALID_ARG;
@@ -57,8 +57,17 @@ extern "C" int lrsa_score_select_static(const lrsa_params_t* params, const void*
   void* scratch = nullptr;
   const int sc = static_scratch(&scratch);
   if (sc != LRSA_OK) return sc;
-  // launch_score_select clears the counters and statistics it needs at zero on the stream before
-  // the kernel; whatever else the previous call left in the array is overwritten before it is read.
-  return launch_score_select(g, static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(V),
-                             idx, score, scratch, static_cast<cudaStream_t>(cuda_stream));
+  // The status word, counters and statistics that must start at zero are cleared on the stream before the
+  // kernel; whatever else the previous call left in the array is overwritten before it is read.
+  return run_score_select(params, g, static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(V),
+                          idx, score, scratch, static_cast<cudaStream_t>(cuda_stream));
+}
+
+// Status word of the last lrsa_score_select_static call on the current device (the first word of the
+// fixed array).  Waits for `cuda_stream`, copies four bytes, allocates nothing.
+extern "C" int lrsa_score_select_static_status(void* cuda_stream) {
+  void* scratch = nullptr;
+  const int sc = static_scratch(&scratch);
+  if (sc != LRSA_OK) return sc;
+  return lrsa_workspace_status(scratch, cuda_stream);
 }

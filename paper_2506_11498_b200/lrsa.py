@@ -28,7 +28,9 @@ class LrsaError(RuntimeError):
 class lrsa_params_t(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("batch", "n_q_heads", "n_kv_heads", "seq_len", "head_dim", "chunk", "lag", "top_k",
-                 "n_sink", "n_dense_prev", "std_ddof")] + [("softmax_scale", ctypes.c_float)]
+                 "n_sink", "n_dense_prev", "std_ddof")] + [("softmax_scale", ctypes.c_float),
+                                                           ("n_seqs", ctypes.c_int32),
+                                                           ("cu_seqlens", ctypes.POINTER(ctypes.c_int32))]
 
 
 @dataclass(frozen=True)
@@ -46,11 +48,18 @@ class Params:
     n_dense_prev: int = 1
     std_ddof: int = 1
     softmax_scale: float = 0.0
+    cu_seqlens: tuple = ()    # packed batch: boundaries (0, ..., seq_len) of the sequences on the token axis
 
     def c(self) -> lrsa_params_t:
-        return lrsa_params_t(self.batch, self.n_q_heads, self.n_kv_heads, self.seq_len, self.head_dim,
-                             self.chunk or self.lag, self.lag, self.top_k, self.n_sink,
-                             self.n_dense_prev, self.std_ddof, self.softmax_scale)
+        cp = lrsa_params_t(self.batch, self.n_q_heads, self.n_kv_heads, self.seq_len, self.head_dim,
+                           self.chunk or self.lag, self.lag, self.top_k, self.n_sink,
+                           self.n_dense_prev, self.std_ddof, self.softmax_scale, 0, None)
+        if self.cu_seqlens:
+            arr = (ctypes.c_int32 * len(self.cu_seqlens))(*self.cu_seqlens)
+            cp.n_seqs = len(self.cu_seqlens) - 1
+            cp.cu_seqlens = ctypes.cast(arr, ctypes.POINTER(ctypes.c_int32))
+            cp._keepalive = arr          # the host array lives as long as the struct
+        return cp
 
     @staticmethod
     def from_workload(w, **kw) -> "Params":
@@ -78,6 +87,8 @@ def lib() -> ctypes.CDLL:
         L.lrsa_attn_fwd.argtypes = [pp, vp, vp, vp, i32p, vp, fp, vp, sz, vp]
         L.lrsa_attn_bwd.argtypes = [pp, vp, vp, vp, vp, vp, fp, i32p, vp, vp, vp, vp, sz, vp]
         L.lrsa_workspace_status.argtypes = [vp, vp]
+        L.lrsa_score_select_static_status.argtypes = [vp]
+        L.lrsa_score_select_static_status.restype = ctypes.c_int
         L.lrsa_status_string.argtypes = [ctypes.c_int]
         L.lrsa_status_string.restype = ctypes.c_char_p
         L.lrsa_last_launch_count.argtypes = []
@@ -154,6 +165,12 @@ def lrsa_score_select_static(params: Params, K, V, idx, score=None, stream=None)
     _check(lib().lrsa_score_select_static(ctypes.byref(cp), _p(K), _p(V), _p(idx), _p(score), _stream(stream)),
            "lrsa_score_select_static")
     return idx, score
+
+
+def lrsa_score_select_static_status(stream=None) -> int:
+    """Status of the last lrsa_score_select_static call on the current device (0 = ok, 5 = a bounded
+    device-side wait expired).  Synchronises the stream."""
+    return lib().lrsa_score_select_static_status(_stream(stream))
 
 
 def lrsa_attn_fwd(params: Params, Q, K, V, idx, O=None, LSE=None, workspace=None, stream=None):

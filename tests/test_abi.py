@@ -80,3 +80,13 @@ def test_geometry_matches_definition():
     for N, S, L, want in ((32768, 4, 1024, 30), (4096, 16, 512, 6), (9, 1, 2, 3), (300, 4, 256, 0), (516, 4, 256, 1)):
         p = lrsa.Params(1, 1, 1, N, 64, L, 1, S)
         assert lrsa.lrsa_num_sel_windows(p) == want
+
+
+def test_packed_parameter_validation():
+    ok = lrsa.Params(**GOOD, cu_seqlens=(0, 300, 1000))
+    assert lrsa.lrsa_num_sel_windows(ok) == ((300 - 4) // 128 - 1) + ((700 - 4) // 128 - 1)
+    for bad in ((1, 300, 1000), (0, 300, 900), (0, 300, 300, 1000), (0, 1200, 1000)):
+        with pytest.raises(lrsa.LrsaError) as e:
+            lrsa.lrsa_num_sel_windows(lrsa.Params(**GOOD, cu_seqlens=bad))
+        assert e.value.status == 1
+    assert lrsa.lrsa_num_sel_windows(lrsa.Params(**{**GOOD, "chunk": 256})) == (1000 - 4) // 128 - 1

@@ -220,3 +220,89 @@ def test_unkept_rows_get_no_gradient_from_later_chunks():
     assert dK[0, 0, un].abs().max().item() == 0 and dV[0, 0, un].abs().max().item() == 0
     assert dV[0, 0, oidx[0, 0, 0]].abs().min(dim=0).values.max().item() > 0
     assert dV[0, 0, : w.S].abs().max().item() > 0
+
+
+# ---- packed variable-length batches and query chunks of several lag windows ----
+
+PACKED_CASES = [
+    # workload (N = last boundary), boundaries, ndp
+    (W("p_two", 1, 4, 2, 1500, 128, 128, 32, 4, seed=51), (0, 4 + 5 * 128 + 77, 1500), 1),     # unequal, both with tails
+    (W("p_three64", 2, 4, 4, 1200, 64, 64, 16, 16, seed=52), (0, 16 + 8 * 64, 16 + 8 * 64 + 10, 1200), 1),  # T = 0; shorter than S
+    (W("p_gqa7", 1, 7, 1, 1000, 128, 100, 30, 3, seed=53, values="channel_offset"), (0, 333, 334, 1000), 1),  # one-token sequence
+    (W("p_ndp0", 1, 2, 2, 900, 64, 128, 32, 4, seed=54), (0, 500, 900), 0),
+]
+
+
+@pytest.mark.parametrize("w,cu,ndp", PACKED_CASES, ids=lambda x: x.name if hasattr(x, "name") else None)
+def test_packed_sequences(w, cu, ndp):
+    """Several sequences back to back on the token axis: every stage against the oracle applied to
+    each sequence on its own."""
+    host = workloads.generate(w)
+    bits = host_bits(host)
+    op = oparams(w, n_dense_prev=ndp)
+    oidx, osc = orc.score_select_packed(op, bits["K"], bits["V"], cu)
+    dev = to_dev(host)
+    p = lrsa.Params.from_workload(w, n_dense_prev=ndp, cu_seqlens=cu)
+    assert lrsa.lrsa_num_sel_windows(p) == oidx.shape[2]
+    sizes = lrsa.lrsa_workspace_bytes(p)
+    ws = [lrsa.new_workspace(s) for s in sizes]
+    idx, sc = lrsa.lrsa_score_select(p, dev["K"], dev["V"], workspace=ws[0], want_score=True)
+    np.testing.assert_allclose(f64(sc), osc, rtol=2e-5, atol=0)
+    got = idx.cpu().numpy()
+    for t0, n, wsel, woff in orc.packed_windows(op, cu):      # per sequence: window numbering restarts
+        if wsel:
+            compare_idx(got[:, :, woff:woff + wsel] - t0, oidx[:, :, woff:woff + wsel] - t0,
+                        osc[:, :, woff:woff + wsel], min(w.S, n), w.L)
+    idx = torch.from_numpy(oidx).cuda()
+    O, LSE = lrsa.lrsa_attn_fwd(p, dev["Q"], dev["K"], dev["V"], idx, workspace=ws[1])
+    dQ, dK, dV = lrsa.lrsa_attn_bwd(p, dev["Q"], dev["K"], dev["V"], O, dev["dO"], LSE, idx, workspace=ws[2])
+    for s in ws:
+        assert lrsa.lrsa_workspace_status(s) == 0
+    oO, oL = orc.attn_fwd_packed(op, bits["Q"], bits["K"], bits["V"], oidx, cu)
+    odQ, odK, odV = orc.attn_bwd_packed(op, bits["Q"], bits["K"], bits["V"], bits["dO"], oidx, cu)
+    check_close("O", f64(O), oO)
+    check_close("LSE", f64(LSE), oL, max_abs=2e-3, rel_l2=1e-4, ulp=0.0)
+    check_close("dQ", f64(dQ), odQ)
+    check_close("dK", f64(dK), odK)
+    check_close("dV", f64(dV), odV)
+
+
+def test_packed_single_sequence_equals_unpacked():
+    w = W("p_one", 1, 4, 2, 4 + 5 * 256 + 77, 128, 256, 64, 4, seed=55)
+    dev = to_dev(workloads.generate(w))
+    a = lrsa.Params.from_workload(w)
+    b = lrsa.Params.from_workload(w, cu_seqlens=(0, w.N))
+    ia, _ = lrsa.lrsa_score_select(a, dev["K"], dev["V"])
+    ib, _ = lrsa.lrsa_score_select(b, dev["K"], dev["V"])
+    assert torch.equal(ia, ib)
+    Oa, La = lrsa.lrsa_attn_fwd(a, dev["Q"], dev["K"], dev["V"], ia)
+    Ob, Lb = lrsa.lrsa_attn_fwd(b, dev["Q"], dev["K"], dev["V"], ia)
+    assert torch.equal(Oa, Ob) and torch.equal(La, Lb)
+
+
+@pytest.mark.parametrize("m", [2, 4])
+def test_query_chunk_of_several_lag_windows(m):
+    """chunk = m * lag: the mask does not depend on how many windows are filled at a time, so the
+    results are those of chunk = lag (and match the oracle, which has no chunk parameter)."""
+    w = W("c_multi", 1, 4, 2, 4 + 6 * 128 + 50, 128, 128, 32, 4, seed=56)
+    host = workloads.generate(w)
+    bits = host_bits(host)
+    op = oparams(w)
+    oidx, _ = orc.score_select(op, bits["K"], bits["V"])
+    oO, _ = orc.attn_fwd(op, bits["Q"], bits["K"], bits["V"], oidx)
+    dev = to_dev(host)
+    p1 = lrsa.Params.from_workload(w)
+    pm = lrsa.Params.from_workload(w, chunk=m * w.L)
+    i1, _ = lrsa.lrsa_score_select(p1, dev["K"], dev["V"])
+    im, _ = lrsa.lrsa_score_select(pm, dev["K"], dev["V"])
+    assert torch.equal(i1, im) and np.array_equal(im.cpu().numpy(), oidx)
+    O1, L1 = lrsa.lrsa_attn_fwd(p1, dev["Q"], dev["K"], dev["V"], i1)
+    Om, Lm = lrsa.lrsa_attn_fwd(pm, dev["Q"], dev["K"], dev["V"], im)
+    assert torch.equal(O1, Om) and torch.equal(L1, Lm)
+    check_close("O", f64(Om), oO)
+    g1 = lrsa.lrsa_attn_bwd(p1, dev["Q"], dev["K"], dev["V"], O1, dev["dO"], L1, i1)
+    gm = lrsa.lrsa_attn_bwd(pm, dev["Q"], dev["K"], dev["V"], Om, dev["dO"], Lm, im)
+    odQ, odK, odV = orc.attn_bwd(op, bits["Q"], bits["K"], bits["V"], bits["dO"], oidx)
+    for name, a, b, ref in zip(("dQ", "dK", "dV"), g1, gm, (odQ, odK, odV)):
+        check_close(name, f64(b), ref)
+        assert (a.float() - b.float()).abs().max().item() <= 2e-2
