@@ -47,9 +47,14 @@ def count_pairs(w, ndp=1) -> int:
     return pairs
 
 
-def flops(w, ndp=1):
-    """Effective FLOPs: 4*d per pair forward (QK^T, PV), 10*d backward (five products)."""
-    p = count_pairs(w, ndp) * w.Hq * w.B
+def flops(w, ndp=1, cu=()):
+    """Effective FLOPs: 4*d per pair forward (QK^T, PV), 10*d backward (five products).  Packed batch:
+    the pairs of every sequence on its own."""
+    if cu:
+        pairs = sum(count_pairs(w.with_(N=b - a, S=min(w.S, b - a)), ndp) for a, b in zip(cu[:-1], cu[1:]))
+    else:
+        pairs = count_pairs(w, ndp)
+    p = pairs * w.Hq * w.B
     return 4 * w.d * p, 10 * w.d * p
 
 
@@ -63,8 +68,10 @@ def measured_peaks():
     if os.path.exists(path):
         m = json.load(open(path))
         return {"hbm_gbs": m["hbm_gbs"], "bf16_tflops": m["bf16_tflops"],
-                "bf16_tflops_sustained": m.get("bf16_tflops_sustained", m["bf16_tflops"]), "source": "measured"}
-    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+                "bf16_tflops_sustained": m.get("bf16_tflops_sustained", m["bf16_tflops"]),
+                "sustained_sm_mhz": (m.get("clocks_under_load") or {}).get("sm_mhz_median"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sustained_sm_mhz": 1300.0,
+            "source": "fallback"}
 
 
 class ClockSampler:
@@ -82,7 +89,7 @@ class ClockSampler:
         try:
             self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(self.index)], stdout=self.file, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -184,8 +191,56 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
-# DRAM bytes per backward call (dK/dV + dQ kernels) from the ncu summary under profiles/, per workload
-BWD_DRAM_BYTES = {"cfg2_32k_gqa7_d128": 3.075e9}
+# DRAM bytes per backward call (dK/dV + dQ kernels) from the ncu summary under profiles/, per workload;
+# empty while the kernels are newer than the last capture (the record then carries null)
+BWD_DRAM_BYTES = {}
+
+
+def spawn_ranks(n: int) -> int:
+    """`python bench.py --gpus N` outside a launcher: start N ranks of this script (one per GPU, NCCL
+    rendezvous on the loopback address) and pass their exit code on.  Rank 0 prints the JSON line."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def parity_sample(w, wl_host, dev_out, idx_dev, n_dense_prev):
+    """A quick look at parity inside the benchmark record: the selection of the timed run against the
+    fp64 CPU checker (windows that differ, all of which must be ties), and the unscaled maximum error of a
+    few sampled rows of O and dQ.  The full comparison lives in tests/; this is a record, not a gate."""
+    import numpy as np
+    from oracle import lrsa_oracle as orc
+    bits = {k: orc.bf16_bits(v) for k, v in wl_host.items()}
+    op = orc.OracleParams(w.B, w.Hq, w.Hkv, w.N, w.d, w.L, w.K, w.S, n_dense_prev=n_dense_prev)
+    oidx, osc = orc.score_select(op, bits["K"], bits["V"])
+    gidx = np.ascontiguousarray(idx_dev.cpu().numpy())
+    differing, not_ties = 0, 0
+    for b in range(w.B):
+        for h in range(w.Hkv):
+            for win in range(oidx.shape[2]):
+                if np.array_equal(gidx[b, h, win], oidx[b, h, win]):
+                    continue
+                differing += 1
+                sc = osc[b, h, win]
+                kth = np.sort(sc)[::-1][w.K - 1]
+                for pos in np.setxor1d(gidx[b, h, win], oidx[b, h, win]):
+                    if abs(sc[pos - w.S - win * w.L] - kth) > 1e-6 * abs(kth):
+                        not_ties += 1
+    rng = np.random.default_rng(7)
+    rows = np.array([[int(rng.integers(0, w.B)), int(rng.integers(0, w.Hq)), int(t)]
+                     for t in (0, w.S + w.L, w.N // 2, w.N - 1)], np.int32)
+    oO, _ = orc.fwd_rows(op, bits["Q"], bits["K"], bits["V"], gidx, rows)
+    odQ = orc.bwd_rows(op, bits["Q"], bits["K"], bits["V"], bits["dO"], gidx, rows)
+    O, dQ = dev_out
+    gO = np.stack([O[b, h, t].float().cpu().numpy() for b, h, t in rows])
+    gdQ = np.stack([dQ[b, h, t].float().cpu().numpy() for b, h, t in rows])
+    return {"idx_windows": int(oidx.shape[0] * oidx.shape[1] * oidx.shape[2]), "idx_windows_differing": differing,
+            "idx_differences_that_are_not_ties": not_ties, "sampled_rows": len(rows),
+            "max_abs_err_O": float(np.abs(gO - oO).max()), "max_abs_err_dQ": float(np.abs(gdQ - odQ).max())}
 
 
 def main():
@@ -198,6 +253,8 @@ def main():
                     help="a configuration name (cfg1_..cfg4_) or a sweep point such as cfg5_L1024_r1/4")
     ap.add_argument("--n-dense-prev", type=int, default=1, choices=[0, 1],
                     help="1: the window before the query chunk is seen uncompressed (the paper); 0: compressed too")
+    ap.add_argument("--cu-seqlens", default="",
+                    help="packed batch: comma-separated boundaries on the token axis, e.g. 0,16384,28672,32768")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -208,6 +265,9 @@ def main():
     if args.impl == "reference":
         run_reference(args, w)
         return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(spawn_ranks(args.gpus))
+    cu = tuple(int(x) for x in args.cu_seqlens.split(",")) if args.cu_seqlens else ()
 
     import torch
     from paper_2506_11498_b200 import lrsa, replicas
@@ -223,7 +283,7 @@ def main():
     # weak scaling: every rank runs its own sequence (independent problems, no data-path collective)
     wl = replicas.rank_workload(w, rank)
     lrsa.lib()
-    p = lrsa.Params.from_workload(wl, n_dense_prev=args.n_dense_prev)
+    p = lrsa.Params.from_workload(wl, n_dense_prev=args.n_dense_prev, cu_seqlens=cu)
     host = {k: v.pin_memory() for k, v in workloads.generate(wl).items()}
     dev = {k: v.cuda(non_blocking=True) for k, v in host.items()}
     ws_sizes = lrsa.lrsa_workspace_bytes(p)
@@ -342,7 +402,7 @@ def main():
             if not torch.equal(outs_host[name], t.cpu()):
                 raise SystemExit(f"end-to-end leg: host copy of {name} differs from the device result")
         e2e_ms = replicas.max_over_ranks(e0.elapsed_time(e1) / n_e2e, dist, "cuda")
-        f_fwd, f_bwd = flops(wl, args.n_dense_prev)
+        f_fwd, f_bwd = flops(wl, args.n_dense_prev, cu)
         e2e = {"value": replicas.job_rate(f_fwd + f_bwd, world, e2e_ms * 1e-3) / 1e12, "unit": UNIT,
                "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "overlap": "uploads, kernels and downloads of consecutive steps overlap (two buffer sets, three streams)"}
@@ -352,12 +412,17 @@ def main():
             dist.destroy_process_group()
         return
 
-    f_fwd, f_bwd = flops(wl, args.n_dense_prev)
+    f_fwd, f_bwd = flops(wl, args.n_dense_prev, cu)
     peaks = measured_peaks()
     med = statistics.median
     bwd_s, fwd_s, score_s = med(t_bwd) * 1e-3, med(t_fwd) * 1e-3, med(t_score) * 1e-3
-    # the kernel is timed inside a long step under the power cap: sustained bf16 peak
-    peak_tf = peaks["bf16_tflops_sustained"]
+    # Which measured peak the kernel is held to: the burst figure when the timed region is short (under a
+    # second) or ran at clocks above those of the sustained measurement, else the sustained one.  Both
+    # fractions are reported; time x clock makes runs at different clocks comparable.
+    timed_s = ms_per_step * 1e-3 * args.steps
+    sm_mhz = (clocks or {}).get("sm_mhz")
+    use_burst = timed_s < 1.0 or bool(sm_mhz and peaks.get("sustained_sm_mhz") and sm_mhz > peaks["sustained_sm_mhz"])
+    peak_tf = peaks["bf16_tflops"] if use_burst else peaks["bf16_tflops_sustained"]
     achieved = f_bwd / bwd_s / 1e12
     line = {
         "metric": METRIC, "value": replicas.job_rate(f_fwd + f_bwd, world, ms_per_step * 1e-3) / 1e12, "unit": UNIT,
@@ -366,10 +431,11 @@ def main():
         "data": "synthetic",
         "config": {"workload": wl.name, "B": wl.B, "N": wl.N, "Hq": wl.Hq, "Hkv": wl.Hkv, "d": wl.d,
                    "L": wl.L, "K": wl.K, "S": wl.S, "values": wl.values, "n_dense_prev": args.n_dense_prev,
+                   "cu_seqlens": list(cu) if cu else None,
                    "l2": "256 MB buffer written between timed steps (outside the per-step events)",
                    "parallelism": f"replicas x{world} (independent sequences, no collective)"},
         "tokens_per_s": world * wl.B * wl.N / (ms_per_step * 1e-3),
-        "pct_of_bf16_peak": {"measured_sustained": 100 * (f_fwd + f_bwd) / (ms_per_step * 1e-3) / 1e12 / peak_tf,
+        "pct_of_bf16_peak": {"measured_sustained": 100 * (f_fwd + f_bwd) / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
                              "measured_burst": 100 * (f_fwd + f_bwd) / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
                              "nominal_2250": 100 * (f_fwd + f_bwd) / (ms_per_step * 1e-3) / 1e12 / 2250.0},
         "stages_ms": {"score_select": med(t_score), "attn_fwd": med(t_fwd), "attn_bwd": med(t_bwd),
@@ -382,14 +448,20 @@ def main():
         # each from an ncu capture; null while the kernels are newer than the last capture.
         "roofline": {"kernel": "lrsa_attn_bwd (lrsa_bwd_dkv_kernel + lrsa_bwd_dq_kernel)", "bound": "tensor",
                      "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
-                     "traffic": BWD_DRAM_BYTES.get(wl.name),
-                     "peak_source": f"{peaks['source']} sustained bf16"},
+                     "frac_burst": achieved / peaks["bf16_tflops"],
+                     "frac_sustained": achieved / peaks["bf16_tflops_sustained"],
+                     "traffic": BWD_DRAM_BYTES.get(wl.name) if not cu else None,
+                     "ms_x_sm_mhz": None if not sm_mhz else med(t_bwd) * sm_mhz,
+                     "peak_source": f"{peaks['source']} {'burst' if use_burst else 'sustained'} bf16 "
+                                    f"(timed region {timed_s:.2f} s at {sm_mhz} MHz)"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches[0] * args.steps,
     }
     if not args.no_cpu_baseline and world == 1:
         s = oracle_sample(w, n_chunks=3, host={k: v for k, v in host.items()} if wl.seed == w.seed else None)
         line["cpu_baseline"] = {"value": s["tflops"], "unit": UNIT, "cores": s["cores"], "kind": "oracle",
                                 "sample": s["sample"]}
+        if not cu:   # packed batches are covered by the tests
+            line["parity_sample"] = parity_sample(wl, host, (O, dQ), idx, args.n_dense_prev)
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
