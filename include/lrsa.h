@@ -166,6 +166,39 @@ int lrsa_attn_bwd(const lrsa_params_t* params, const void* Q, const void* K, con
                   void* dK, void* dV, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Inference side (Section 3.2: the KV-cache update of Attn-Fill 1 / Attn-Fill 2; its last paragraph: the mask
+ * does not depend on the query, so the KV cache can be condensed physically).  The cache is one caller-owned
+ * device buffer of lrsa_cache_bytes bytes per layer (256-byte aligned, contents managed by these calls).  Per
+ * (batch, KV head) it holds the sink rows, top_k kept rows of every compressed window, and a ring of 2*lag rows
+ * with the uncompressed recent tokens: S + W*K + 2L rows instead of seq_len.  seq_len is the capacity in tokens.
+ * Only n_dense_prev = 1 and unpacked batches are supported (LRSA_ERR_UNSUPPORTED otherwise).
+ *
+ * lrsa_cache_append adds the tokens n_prev .. n_prev + n_new - 1 (n_prev = tokens already in the cache; the caller
+ * keeps that count; the first call has n_prev = 0).  When the first token of query chunk c arrives, window c-2 is
+ * scored with window c-1 as its reference (Eq. 4-8, the arithmetic of lrsa_score_select), its top_k rows are
+ * appended to the kept rows and it leaves the ring; until then the queries of chunk c-1 see it whole, as the
+ * mask of Section 3.2 prescribes.  Any n_new is accepted.
+ *   k_new, v_new in : bf16 [B, Hkv, n_new, d]
+ *
+ * lrsa_attn_decode: Eq. 3 for ONE query token per (batch, query head), the token at position n_tokens - 1 of a
+ * cache that holds n_tokens tokens; it sees exactly what row n_tokens - 1 of lrsa_attn_fwd sees.  fp32 arithmetic.
+ *   q in : bf16 [B, Hq, d];  o out : bf16 [B, Hq, d];  lse out (optional) : fp32 [B, Hq]
+ *
+ * lrsa_cache_kept returns a device pointer into the cache: int32 [B, Hkv, w_cap, top_k], the kept positions of the
+ * windows compressed so far (rows of later windows are undefined).
+ * `workspace` (lrsa_cache_bytes' second figure) is scratch for both calls; its status word is read with
+ * lrsa_workspace_status.
+ */
+int lrsa_cache_bytes(const lrsa_params_t* params, size_t* cache_bytes, size_t* workspace_bytes);
+int lrsa_cache_append(const lrsa_params_t* params, void* cache, size_t cache_bytes, const void* k_new,
+                      const void* v_new, int32_t n_prev, int32_t n_new, void* workspace, size_t workspace_bytes,
+                      void* cuda_stream);
+int lrsa_cache_kept(const lrsa_params_t* params, const void* cache, const int32_t** idx, int32_t* w_cap);
+int lrsa_attn_decode(const lrsa_params_t* params, const void* cache, size_t cache_bytes, const void* q,
+                     int32_t n_tokens, void* o, float* lse, void* workspace, size_t workspace_bytes,
+                     void* cuda_stream);
+
+/*
  * Reads the status word that the last call using `workspace` left there.  Synchronises
  * `cuda_stream`.  Returns LRSA_OK, LRSA_ERR_TIMEOUT, or LRSA_ERR_CUDA if the copy failed.
  */

@@ -38,7 +38,7 @@ int make_geom(const lrsa_params_t* p, Geom* g) {
   g->C = g->W + (g->T > 0 ? 1 : 0);
   g->Wsel = g->W > 1 ? g->W - 1 : 0;
   g->Rc = g->S + g->Wsel * g->K;
-  g->Nrow = g->N; g->tok0 = 0; g->Wtot = g->Wsel; g->woff = 0;
+  g->Nrow = g->N; g->tok0 = 0; g->Wtot = g->Wsel; g->woff = 0; g->emit_off = 0; g->win_stride = g->L;
   if (p->n_seqs < 0) return LRSA_ERR_INVALID_ARG;
   if (p->n_seqs > 0) {
     if (!p->cu_seqlens || p->cu_seqlens[0] != 0 || p->cu_seqlens[p->n_seqs] != p->seq_len) return LRSA_ERR_INVALID_ARG;
@@ -61,6 +61,7 @@ void seq_geom(const Geom& whole, const int32_t* cu, int n_seqs, int s, int woff,
   if (n_seqs <= 0 || !cu) return;   // the whole row is the one sequence
   Geom& g = *out;
   g.tok0 = cu[s];
+  g.emit_off = cu[s];
   g.N = cu[s + 1] - cu[s];
   g.S = whole.S < g.N ? whole.S : g.N;   // a sequence shorter than the sink count is all sinks
   g.W = (g.N - g.S) / g.L;

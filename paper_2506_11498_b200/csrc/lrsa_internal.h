@@ -25,6 +25,9 @@ struct Geom {
   // The launchers shift every tensor pointer by tok0 tokens and use Nrow as the row stride, so the
   // kernels see an ordinary sequence; kept positions (idx) stay positions in the whole row.
   int Nrow, tok0, Wtot, woff;
+  // Scoring only: value added to the positions written to idx (tok0 unless the rows are a ring buffer)
+  // and distance in tokens from window w to window w+1 (L unless the rows are a ring buffer).
+  int emit_off, win_stride;
 };
 
 // Sequence s of a packed batch (cu = boundaries, n_seqs + 1 entries) as a Geom of its own.

@@ -37,9 +37,11 @@ struct ScoreArgs {
   uint32_t* mm;   // [BH, W, 2 (K,V), 2 (min,max), d] order-preserving keys, zero = identity
   float* spread;  // [BH, Wsel, 2 (K,V), L]
   int BH, N, L, Kk, S, W, Wsel, n_slices, ddof;   // N: tokens per (batch, head) row of K and V (the row stride)
-  int tok0, Wtot, woff;   // packed batches: K and V point at token tok0 of the rows; this sequence's windows are
-                          // [woff, woff + Wsel) of the Wtot windows per head of idx and score; positions are emitted + tok0
-  size_t elems;           // elements of K (and of V) from the shifted pointer to the end of the tensor
+  int tok0, Wtot, woff;   // the sequence starts at token tok0 of the rows; its windows are [woff, woff + Wsel) of the
+                          // Wtot windows per head of idx and score
+  int emit_off;           // added to S + w*L + i when a position is written to idx
+  int win_stride;         // tokens from window w to window w+1 in memory (L; -L or L for a two-window ring buffer)
+  long long elems;        // elements of K (and of V)
   int spin_limit;
 };
 
@@ -195,7 +197,7 @@ __device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* 
   // emit kept positions in ascending order: every thread takes a run of consecutive tokens, one block
   // scan gives the number of kept tokens before the run
   int32_t* out = a.idx + (size_t)(bh * a.Wtot + a.woff + w) * a.Kk;
-  const int pos0 = a.tok0 + a.S + w * L;   // position of the window's first token in the row
+  const int pos0 = a.emit_off + a.S + w * L;   // position of the window's first token
   const int per = (L + kThreads - 1) / kThreads;
   const int i_lo = min(L, tid * per), i_hi = min(L, i_lo + per);
   int packed = 0;   // tokens above the K-th score | tokens equal to it << 16
@@ -250,13 +252,13 @@ __global__ void __launch_bounds__(kThreads) score_select_kernel(const ScoreArgs 
   // the slice of K and of V, held in registers for both phases
   uint4 kq[kSteps], vq[kSteps];
   bool valid[kSteps];
-  const size_t row0 = (size_t)bh * a.N + a.S + (size_t)w * a.L;
+  const long long row0 = (long long)bh * a.N + a.tok0 + a.S + (long long)w * a.win_stride;
 #pragma unroll
   for (int s = 0; s < kSteps; ++s) {
     const int i = slice * TOK + s * RPS + row;
     valid[s] = i < a.L;
     if (valid[s]) {
-      const size_t off = (row0 + i) * D + chunk * 8;
+      const long long off = (row0 + i) * D + chunk * 8;
       kq[s] = __ldcs(reinterpret_cast<const uint4*>(a.K + off));
       vq[s] = __ldcs(reinterpret_cast<const uint4*>(a.V + off));
     } else {
@@ -482,12 +484,12 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
       if (*abort) break;
       const int rows = min(TOK, a.L - slice * TOK);
       const uint32_t bytes = (uint32_t)rows * D * 2;
-      const size_t off = ((size_t)bh * a.N + a.S + (size_t)w * a.L + (size_t)slice * TOK) * D;
+      const long long off = ((long long)bh * a.N + a.tok0 + a.S + (long long)w * a.win_stride + (long long)slice * TOK) * D;
       const uint32_t bar = ptx::smem_u32(&full_bar[slot]);
       const uint32_t dst = ptx::smem_u32(smem + slot * kStageBytes);
       // self-check: the slice lies inside the tensor and the copy is 16-byte granular; otherwise give up
       // (status word) instead of issuing it
-      if (w < 0 || w >= a.W || rows <= 0 || off + (size_t)rows * D > a.elems || (bytes & 15u) ||
+      if (w < 0 || w >= a.W || rows <= 0 || off < 0 || off + (long long)rows * D > a.elems || (bytes & 15u) ||
           ((reinterpret_cast<uintptr_t>(a.K + off) | reinterpret_cast<uintptr_t>(a.V + off) | dst) & 15u)) {
         *abort = 1;
         atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT);
@@ -746,16 +748,15 @@ int launch_score_select(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat
     launch_counter().n++;
   }
   ScoreArgs a;
-  // the sequence starts at token tok0 of every row: shift the inputs, keep the row stride
-  a.K = K + (size_t)g.tok0 * g.d; a.V = V + (size_t)g.tok0 * g.d; a.idx = idx; a.score = score;
+  a.K = K; a.V = V; a.idx = idx; a.score = score;
   a.hdr = reinterpret_cast<WsHeader*>(base);
   a.ready = reinterpret_cast<int*>(base + lay.ready);
   a.done = reinterpret_cast<int*>(base + lay.done);
   a.mm = reinterpret_cast<uint32_t*>(base + lay.mm);
   a.spread = reinterpret_cast<float*>(base + lay.spread);
   a.BH = g.B * g.Hkv; a.N = g.Nrow; a.L = g.L; a.Kk = g.K; a.S = g.S; a.W = g.W; a.Wsel = g.Wsel;
-  a.tok0 = g.tok0; a.Wtot = g.Wtot; a.woff = g.woff;
-  a.elems = ((size_t)g.B * g.Hkv * g.Nrow - (size_t)g.tok0) * g.d;
+  a.tok0 = g.tok0; a.Wtot = g.Wtot; a.woff = g.woff; a.emit_off = g.emit_off; a.win_stride = g.win_stride;
+  a.elems = (long long)g.B * g.Hkv * g.Nrow * g.d;
   a.ddof = g.ddof;
   a.spin_limit = 1 << 21;
   const int tok = g.d == 128 ? tok_per_unit<128>() : tok_per_unit<64>();

@@ -86,6 +86,13 @@ def lib() -> ctypes.CDLL:
         L.lrsa_score_select_static.restype = ctypes.c_int
         L.lrsa_attn_fwd.argtypes = [pp, vp, vp, vp, i32p, vp, fp, vp, sz, vp]
         L.lrsa_attn_bwd.argtypes = [pp, vp, vp, vp, vp, vp, fp, i32p, vp, vp, vp, vp, sz, vp]
+        i32 = ctypes.c_int32
+        L.lrsa_cache_bytes.argtypes = [pp, ctypes.POINTER(sz), ctypes.POINTER(sz)]
+        L.lrsa_cache_append.argtypes = [pp, vp, sz, vp, vp, i32, i32, vp, sz, vp]
+        L.lrsa_cache_kept.argtypes = [pp, vp, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(i32)]
+        L.lrsa_attn_decode.argtypes = [pp, vp, sz, vp, i32, vp, fp, vp, sz, vp]
+        for name in ("lrsa_cache_bytes", "lrsa_cache_append", "lrsa_cache_kept", "lrsa_attn_decode"):
+            getattr(L, name).restype = ctypes.c_int
         L.lrsa_workspace_status.argtypes = [vp, vp]
         L.lrsa_score_select_static_status.argtypes = [vp]
         L.lrsa_score_select_static_status.restype = ctypes.c_int
@@ -214,3 +221,57 @@ def lrsa_last_launch_count() -> int:
 
 def lrsa_debug_set_impl(impl: int):
     _check(lib().lrsa_debug_set_impl(int(impl)), "lrsa_debug_set_impl")
+
+
+class KVCache:
+    """Condensed KV cache of one layer for inference (Section 3.2): owns the device buffer and the token
+    count; every operation runs in the library's kernels."""
+
+    def __init__(self, params: Params, device="cuda"):
+        self.params = params
+        a, b = ctypes.c_size_t(0), ctypes.c_size_t(0)
+        cp = params.c()
+        _check(lib().lrsa_cache_bytes(ctypes.byref(cp), ctypes.byref(a), ctypes.byref(b)), "lrsa_cache_bytes")
+        self.buf = torch.zeros(a.value, dtype=torch.uint8, device=device)
+        self.ws = new_workspace(b.value, device)
+        self.n_tokens = 0
+
+    def append(self, k_new, v_new, stream=None):
+        """k_new, v_new: bf16 [B, Hkv, n_new, d] (contiguous)."""
+        n_new = k_new.shape[2]
+        cp = self.params.c()
+        _check(lib().lrsa_cache_append(ctypes.byref(cp), _p(self.buf), self.buf.numel(), _p(k_new), _p(v_new),
+                                       self.n_tokens, n_new, _p(self.ws), self.ws.numel(), _stream(stream)),
+               "lrsa_cache_append")
+        self.n_tokens += n_new
+
+    def decode(self, q, o=None, lse=None, stream=None):
+        """q: bf16 [B, Hq, d], the query of the last token in the cache.  Returns (o, lse)."""
+        if o is None:
+            o = torch.empty_like(q)
+        if lse is None:
+            lse = torch.empty(q.shape[:2], dtype=torch.float32, device=q.device)
+        cp = self.params.c()
+        _check(lib().lrsa_attn_decode(ctypes.byref(cp), _p(self.buf), self.buf.numel(), _p(q), self.n_tokens, _p(o),
+                                      _p(lse), _p(self.ws), self.ws.numel(), _stream(stream)), "lrsa_attn_decode")
+        return o, lse
+
+    def kept(self):
+        """int32 [B, Hkv, w_cap, top_k] view of the kept positions (windows compressed so far are valid)."""
+        ptr, wcap = ctypes.c_void_p(0), ctypes.c_int32(0)
+        cp = self.params.c()
+        _check(lib().lrsa_cache_kept(ctypes.byref(cp), _p(self.buf), ctypes.byref(ptr), ctypes.byref(wcap)),
+               "lrsa_cache_kept")
+        off = ptr.value - self.buf.data_ptr()
+        n = self.params.batch * self.params.n_kv_heads * wcap.value * self.params.top_k
+        return self.buf[off:off + 4 * n].view(torch.int32).view(self.params.batch, self.params.n_kv_heads, wcap.value,
+                                                                 self.params.top_k)
+
+    def windows_compressed(self) -> int:
+        p = self.params
+        if self.n_tokens <= p.n_sink:
+            return 0
+        return max((self.n_tokens - 1 - p.n_sink) // p.lag - 1, 0)
+
+    def status(self, stream=None) -> int:
+        return lrsa_workspace_status(self.ws, stream)
