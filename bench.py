@@ -208,6 +208,38 @@ def spawn_ranks(n: int) -> int:
     return subprocess.call(cmd)
 
 
+def decode_leg(lrsa, torch, wl, p, dev, flush, peaks):
+    """Inference side of the same layer: the condensed cache is filled with the workload's K/V, then one
+    decode step (the query of the last token over sinks + kept rows + ring) is timed with L2 flushed, and
+    one cache growth step of a whole lag window (which scores and condenses one window)."""
+    cache = lrsa.KVCache(p)
+    n0 = wl.N - wl.L - 1                      # leave room for one more window of growth
+    cache.append(dev["K"][:, :, :n0].contiguous(), dev["V"][:, :, :n0].contiguous())
+    q = dev["Q"][:, :, n0 - 1].contiguous()
+    o = torch.empty_like(q)
+    lse = torch.empty(q.shape[:2], dtype=torch.float32, device="cuda")
+    ts = []
+    for i in range(13):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); cache.decode(q, o, lse); e1.record(); torch.cuda.synchronize()
+        if i >= 3:
+            ts.append(e0.elapsed_time(e1))
+    c = (n0 - 1 - wl.S) // wl.L
+    keys = wl.S + max(c - 1, 0) * wl.K + (n0 - 1 - (wl.S + max(c - 1, 0) * wl.L) + 1)
+    nbytes = wl.B * wl.Hkv * keys * wl.d * 2 * 2
+    ms = statistics.median(ts)
+    kn = dev["K"][:, :, n0:n0 + wl.L].contiguous(); vn = dev["V"][:, :, n0:n0 + wl.L].contiguous()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    flush.zero_(); e0.record(); cache.append(kn, vn); e1.record(); torch.cuda.synchronize()
+    if cache.status() != 0:
+        raise SystemExit("decode leg: the cache workspace reports a timeout")
+    return {"tokens_in_cache": n0, "keys_per_kv_head": keys, "cache_rows_per_kv_head": wl.S + max(c - 1, 0) * wl.K + 2 * wl.L,
+            "decode_us": ms * 1e3, "decode_gbs": nbytes / (ms * 1e-3) / 1e9,
+            "decode_frac_of_hbm": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "append_one_window_us": e0.elapsed_time(e1) * 1e3}
+
+
 def parity_sample(w, wl_host, dev_out, idx_dev, n_dense_prev):
     """A quick look at parity inside the benchmark record: the selection of the timed run against the
     fp64 CPU checker (windows that differ, all of which must be ties), and the unscaled maximum error of a
@@ -257,6 +289,7 @@ def main():
                     help="packed batch: comma-separated boundaries on the token axis, e.g. 0,16384,28672,32768")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-decode", action="store_true", help="skip the inference-side leg (condensed cache + decode)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -456,6 +489,8 @@ def main():
                                     f"(timed region {timed_s:.2f} s at {sm_mhz} MHz)"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches[0] * args.steps,
     }
+    if not args.no_decode and world == 1 and not cu and args.n_dense_prev == 1:
+        line["decode"] = decode_leg(lrsa, torch, wl, p, dev, flush, peaks)
     if not args.no_cpu_baseline and world == 1:
         s = oracle_sample(w, n_chunks=3, host={k: v for k, v in host.items()} if wl.seed == w.seed else None)
         line["cpu_baseline"] = {"value": s["tflops"], "unit": UNIT, "cores": s["cores"], "kind": "oracle",

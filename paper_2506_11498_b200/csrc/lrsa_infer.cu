@@ -15,6 +15,7 @@
 // (HBM-bound: 4*d bytes per key, a few FMAs per byte): the keys are split over CTAs, every warp keeps an
 // online softmax per query head, and a second small kernel merges the partial results.
 #include "lrsa_internal.h"
+#include "sm100_ptx.h"
 
 namespace lrsa {
 namespace {
@@ -86,38 +87,89 @@ __global__ void cache_keep_kernel(const int32_t* __restrict__ idx, const __nv_bf
 
 
 // ---- decode attention ----
-constexpr int kDecThreads = 256;
+constexpr int kDecThreads = 128;
 constexpr int kDecHeads = 8;      // query heads of a group handled per pass over the keys
+constexpr int kDecKeys = 128;     // keys per CTA, staged in shared memory by bulk copies
 
 struct DecodeArgs {
   const __nv_bfloat16 *q, *k_list, *v_list, *k_ring, *v_ring;
   float* part;          // [BHkv][n_split][G][D + 2]: unnormalised output, running maximum (log2 domain), sum
+  int* status;          // workspace status word
   int BHkv, Hq, Hkv, G, rows_list, L, S;
   int n_list, n_ring, ring0;   // keys: list rows [0, n_list), then n_ring ring rows starting at ring row ring0
-  int n_split, per_split;
+  int n_split;
   float scale_log2;
 };
 
 __device__ __forceinline__ float bf_lo(uint32_t p) { return __uint_as_float(p << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t p) { return __uint_as_float(p & 0xffff0000u); }
 
-// Grid (n_split, BHkv).  D/8 lanes share a key (16 bytes each), so a warp works on 32/(D/8) keys at a time;
-// every such lane group keeps an online softmax (maximum, sum, 8 output channels per lane) per query head.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// Grid (n_split, BHkv).  The CTA's (at most) 128 keys are runs of consecutive rows of the list and of the
+// ring (at most three runs: the ring wraps once); one thread fetches K and V of every run with bulk copies,
+// so all of the CTA's bytes are in flight at once.  Then D/8 lanes share a key (16 bytes each), a warp works
+// on 32/(D/8) keys at a time, and every such lane group keeps an online softmax (maximum, sum, 8 output
+// channels per lane) per query head.
 template <int D>
 __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const DecodeArgs a) {
   constexpr int LPK = D / 8, KPW = 32 / LPK;           // lanes per key, keys per warp step
   constexpr int kGroups = (kDecThreads / 32) * KPW;    // lane groups per CTA
+  extern __shared__ __align__(128) unsigned char dec_smem[];   // K rows [kDecKeys][D], then V rows
+  __shared__ __align__(8) uint64_t bar;
   __shared__ float red_m[kGroups][kDecHeads], red_l[kGroups][kDecHeads];
   __shared__ float red_o[kGroups][D];
+  __shared__ int s_fail;
   const int bh = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane / LPK, ch = (lane % LPK) * 8, grp = warp * KPW + sub;
   const int n_keys = a.n_list + a.n_ring;
-  const int k_lo = split * a.per_split, k_hi = min(n_keys, k_lo + a.per_split);
+  const int k_lo = split * kDecKeys, k_hi = min(n_keys, k_lo + kDecKeys), nk = k_hi - k_lo;
   const int b = bh / a.Hkv, hkv = bh % a.Hkv;
-  const __nv_bfloat16* kl = a.k_list + (size_t)bh * a.rows_list * D;
-  const __nv_bfloat16* vl = a.v_list + (size_t)bh * a.rows_list * D;
-  const __nv_bfloat16* kr = a.k_ring + (size_t)bh * 2 * a.L * D;
-  const __nv_bfloat16* vr = a.v_ring + (size_t)bh * 2 * a.L * D;
+  __nv_bfloat16* sK = reinterpret_cast<__nv_bfloat16*>(dec_smem);
+  __nv_bfloat16* sV = sK + kDecKeys * D;
+  if (tid == 0) {
+    s_fail = 0;
+    ptx::mbar_init(ptx::smem_u32(&bar), 1);
+    ptx::fence_barrier_init();
+    ptx::mbar_expect_tx(ptx::smem_u32(&bar), (uint32_t)nk * D * 2 * 2);
+    const __nv_bfloat16* kl = a.k_list + (size_t)bh * a.rows_list * D;
+    const __nv_bfloat16* vl = a.v_list + (size_t)bh * a.rows_list * D;
+    const __nv_bfloat16* kr = a.k_ring + (size_t)bh * 2 * a.L * D;
+    const __nv_bfloat16* vr = a.v_ring + (size_t)bh * 2 * a.L * D;
+    int i = k_lo;
+    while (i < k_hi) {
+      const __nv_bfloat16 *ks, *vs;
+      int run;
+      if (i < a.n_list) {
+        run = min(k_hi, a.n_list) - i;
+        ks = kl + (size_t)i * D; vs = vl + (size_t)i * D;
+      } else {
+        const int r = (a.ring0 + (i - a.n_list)) % (2 * a.L);
+        run = min(k_hi - i, 2 * a.L - r);
+        ks = kr + (size_t)r * D; vs = vr + (size_t)r * D;
+      }
+      const uint32_t bytes = (uint32_t)run * D * 2;
+      bulk_load(ptx::smem_u32(sK + (size_t)(i - k_lo) * D), ks, bytes, ptx::smem_u32(&bar));
+      bulk_load(ptx::smem_u32(sV + (size_t)(i - k_lo) * D), vs, bytes, ptx::smem_u32(&bar));
+      i += run;
+    }
+  }
+  __syncthreads();
+  {
+    // bounded wait for the copies; a CTA that gives up records it and leaves its partial result empty
+    bool ok = ptx::mbar_try_wait(ptx::smem_u32(&bar), 0);
+    const long long t0 = clock64();
+    while (!ok) {
+      ok = ptx::mbar_try_wait(ptx::smem_u32(&bar), 0);
+      if (!ok && clock64() - t0 > 4000000000LL) { s_fail = 1; break; }
+    }
+  }
+  __syncthreads();
+  const bool failed = s_fail != 0;
+  if (failed && tid == 0) atomicExch(a.status, (int)LRSA_ERR_TIMEOUT);
 
   for (int g0 = 0; g0 < a.G; g0 += kDecHeads) {
     const int ng = min(kDecHeads, a.G - g0);
@@ -134,20 +186,13 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const Decod
         for (int e = 0; e < 4; ++e) { q[g][2 * e] = bf_lo(w[e]) * a.scale_log2; q[g][2 * e + 1] = bf_hi(w[e]) * a.scale_log2; }
       }
     }
-    for (int i0 = k_lo + warp * KPW; i0 < k_hi; i0 += (kDecThreads / 32) * KPW) {
+    for (int i0 = warp * KPW; i0 < nk && !failed; i0 += (kDecThreads / 32) * KPW) {
       const int i = i0 + sub;
-      const bool live = i < k_hi;
+      const bool live = i < nk;
       uint4 kx = make_uint4(0, 0, 0, 0), vx = make_uint4(0, 0, 0, 0);
       if (live) {
-        const __nv_bfloat16 *kp, *vp;
-        if (i < a.n_list) {
-          kp = kl + (size_t)i * D; vp = vl + (size_t)i * D;
-        } else {
-          const int r = (a.ring0 + (i - a.n_list)) % (2 * a.L);
-          kp = kr + (size_t)r * D; vp = vr + (size_t)r * D;
-        }
-        kx = *reinterpret_cast<const uint4*>(kp + ch);
-        vx = *reinterpret_cast<const uint4*>(vp + ch);
+        kx = *reinterpret_cast<const uint4*>(sK + (size_t)i * D + ch);
+        vx = *reinterpret_cast<const uint4*>(sV + (size_t)i * D + ch);
       }
       const uint32_t kw[4] = {kx.x, kx.y, kx.z, kx.w}, vw[4] = {vx.x, vx.y, vx.z, vx.w};
       float kf[8], vf[8];
@@ -199,35 +244,46 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const Decod
   }
 }
 
-// One CTA of D threads per (batch, query head): merges the partial results of the splits.
+// One CTA per (batch, query head): merges the partial results of the splits.  kMergeRows thread rows take
+// alternate splits (so their loads are in flight together), then the rows are merged through shared memory.
+constexpr int kMergeRows = 8;
 template <int D>
-__global__ void decode_merge_kernel(const float* __restrict__ part, __nv_bfloat16* __restrict__ o, float* __restrict__ lse,
-                                    int Hq, int Hkv, int G, int n_split) {
-  const int bhq = blockIdx.x, b = bhq / Hq, hq = bhq % Hq, hkv = hq / G, g = hq % G, c = threadIdx.x;
+__global__ void __launch_bounds__(kMergeRows * D) decode_merge_kernel(const float* __restrict__ part,
+                                                                       __nv_bfloat16* __restrict__ o,
+                                                                       float* __restrict__ lse, int Hq, int Hkv, int G,
+                                                                       int n_split) {
+  __shared__ float sm_m[kMergeRows], sm_l[kMergeRows], sm_o[kMergeRows][D];
+  const int bhq = blockIdx.x, b = bhq / Hq, hq = bhq % Hq, hkv = hq / G, g = hq % G;
+  const int c = threadIdx.x % D, row = threadIdx.x / D;
   const float* base = part + (((size_t)(b * Hkv + hkv) * n_split) * G + g) * (D + 2);
   const size_t stride = (size_t)G * (D + 2);
-  float M = -INFINITY;
-  for (int s = 0; s < n_split; ++s) M = fmaxf(M, base[s * stride + D]);
-  float acc = 0.f, l = 0.f;
-  for (int s = 0; s < n_split; ++s) {
+  float M = -INFINITY, acc = 0.f, l = 0.f;
+  for (int s = row; s < n_split; s += kMergeRows) {
     const float ms = base[s * stride + D];
-    const float f = ms == -INFINITY ? 0.f : exp2f(ms - M);
-    acc = fmaf(base[s * stride + c], f, acc);
-    l = fmaf(base[s * stride + D + 1], f, l);
+    if (ms == -INFINITY) continue;
+    const float mn = fmaxf(M, ms), f0 = exp2f(M - mn), f1 = exp2f(ms - mn);
+    acc = acc * f0 + base[s * stride + c] * f1;
+    l = l * f0 + base[s * stride + D + 1] * f1;
+    M = mn;
   }
-  o[(size_t)bhq * D + c] = __float2bfloat16(acc / l);
-  if (c == 0 && lse) lse[bhq] = (M + log2f(l)) * 0.6931471805599453f;
+  sm_o[row][c] = acc;
+  if (c == 0) { sm_m[row] = M; sm_l[row] = l; }
+  __syncthreads();
+  if (row == 0) {
+    float Mt = -INFINITY;
+    for (int r = 0; r < kMergeRows; ++r) Mt = fmaxf(Mt, sm_m[r]);
+    float at = 0.f, lt = 0.f;
+    for (int r = 0; r < kMergeRows; ++r) {
+      const float f = sm_m[r] == -INFINITY ? 0.f : exp2f(sm_m[r] - Mt);
+      at = fmaf(sm_o[r][c], f, at);
+      lt = fmaf(sm_l[r], f, lt);
+    }
+    o[(size_t)bhq * D + c] = __float2bfloat16(at / lt);
+    if (c == 0 && lse) lse[bhq] = (Mt + log2f(lt)) * 0.6931471805599453f;
+  }
 }
 
-int decode_splits(const Geom& g, int n_keys, int* per_split) {
-  const int BH = g.B * g.Hkv;
-  int want = (2 * 148 + BH - 1) / BH;               // about two CTAs per SM over all heads
-  const int by_len = (n_keys + 127) / 128;          // at least 128 keys per CTA
-  int n = want < by_len ? want : by_len;
-  if (n < 1) n = 1;
-  *per_split = (n_keys + n - 1) / n;
-  return (n_keys + *per_split - 1) / *per_split;
-}
+int decode_splits(int n_keys) { return n_keys > 0 ? (n_keys + kDecKeys - 1) / kDecKeys : 1; }
 
 }  // namespace
 }  // namespace lrsa
@@ -247,7 +303,8 @@ int lrsa_cache_bytes(const lrsa_params_t* params, size_t* cache_bytes, size_t* w
     Geom two = g;
     two.N = two.Nrow = 2 * g.L; two.S = 0; two.W = 2; two.Wsel = 1; two.T = 0; two.C = 2;
     const size_t a = score_select_ws_bytes(two);
-    const size_t b = 256 + (size_t)g.B * g.Hkv * (2 * 148 + 1) * g.G * (g.d + 2) * sizeof(float);
+    // a sequence of N tokens never shows a query more than S + Wcap*K + 2L keys
+    const size_t b = 256 + (size_t)g.B * g.Hkv * decode_splits(cache_layout(g).rows_list + 2 * g.L) * g.G * (g.d + 2) * sizeof(float);
     *workspace_bytes = a > b ? a : b;
   }
   return LRSA_OK;
@@ -367,17 +424,26 @@ int lrsa_attn_decode(const lrsa_params_t* params, const void* cache, size_t cach
     a.n_ring = t - (g.S + nc * g.L) + 1;
     a.ring0 = (nc * g.L) % (2 * g.L);
   }
-  a.n_split = decode_splits(g, a.n_list + a.n_ring, &a.per_split);
+  a.n_split = decode_splits(a.n_list + a.n_ring);
   a.scale_log2 = g.scale * 1.4426950408889634f;
+  a.status = &reinterpret_cast<WsHeader*>(workspace)->status;
+  LRSA_CUDA_CHECK(cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st));
+  launch_counter().n++;
   const dim3 grid(a.n_split, a.BHkv);
-  if (g.d == 128) decode_partial_kernel<128><<<grid, kDecThreads, 0, st>>>(a);
-  else decode_partial_kernel<64><<<grid, kDecThreads, 0, st>>>(a);
+  const size_t smem = (size_t)2 * kDecKeys * g.d * sizeof(__nv_bfloat16);
+  if (g.d == 128) {
+    LRSA_CUDA_CHECK(cudaFuncSetAttribute(decode_partial_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    decode_partial_kernel<128><<<grid, kDecThreads, smem, st>>>(a);
+  } else {
+    LRSA_CUDA_CHECK(cudaFuncSetAttribute(decode_partial_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    decode_partial_kernel<64><<<grid, kDecThreads, smem, st>>>(a);
+  }
   LRSA_CUDA_CHECK(cudaGetLastError());
   launch_counter().n++;
   if (g.d == 128)
-    decode_merge_kernel<128><<<g.B * g.Hq, 128, 0, st>>>(a.part, static_cast<__nv_bfloat16*>(o), lse, g.Hq, g.Hkv, g.G, a.n_split);
+    decode_merge_kernel<128><<<g.B * g.Hq, kMergeRows * 128, 0, st>>>(a.part, static_cast<__nv_bfloat16*>(o), lse, g.Hq, g.Hkv, g.G, a.n_split);
   else
-    decode_merge_kernel<64><<<g.B * g.Hq, 64, 0, st>>>(a.part, static_cast<__nv_bfloat16*>(o), lse, g.Hq, g.Hkv, g.G, a.n_split);
+    decode_merge_kernel<64><<<g.B * g.Hq, kMergeRows * 64, 0, st>>>(a.part, static_cast<__nv_bfloat16*>(o), lse, g.Hq, g.Hkv, g.G, a.n_split);
   LRSA_CUDA_CHECK(cudaGetLastError());
   launch_counter().n++;
   return LRSA_OK;
