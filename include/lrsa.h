@@ -217,6 +217,14 @@ int lrsa_last_launch_count(void);
  */
 int lrsa_debug_set_impl(int impl);
 
+/*
+ * Test hook (process-wide) for the bounded device-side wait of the scoring kernel that handles lag windows
+ * beyond 4096 tokens: the number of polls a work unit grants the statistics of the following window.  A
+ * negative value makes that wait give up at once, so that the LRSA_ERR_TIMEOUT path can be exercised without
+ * wedging a kernel (the call then leaves idx undefined and the status word set); 0 restores the default.
+ */
+int lrsa_debug_set_wait_limit(int polls);
+
 #ifdef __cplusplus
 }
 #endif

@@ -74,14 +74,18 @@ void seq_geom(const Geom& whole, const int32_t* cu, int n_seqs, int s, int woff,
 
 int run_score_select(const lrsa_params_t* p, const Geom& whole, const __nv_bfloat16* K, const __nv_bfloat16* V,
                      int32_t* idx, float* score, void* ws, cudaStream_t st) {
-  LRSA_CUDA_CHECK(cudaMemsetAsync(ws, 0, sizeof(WsHeader), st));
-  launch_counter().n++;
   const int n_seqs = geom_n_seqs(p);
+  // one sequence scored by the kernel that clears the status word itself: a single launch
+  const bool in_kernel = n_seqs == 1 && score_select_clears_status(whole);
+  if (!in_kernel) {
+    LRSA_CUDA_CHECK(cudaMemsetAsync(ws, 0, sizeof(WsHeader), st));
+    launch_counter().n++;
+  }
   int woff = 0;
   for (int s = 0; s < n_seqs; ++s) {
     Geom g;
     seq_geom(whole, p->cu_seqlens, p->n_seqs, s, woff, &g);
-    const int rc = launch_score_select(g, K, V, idx, score, ws, st);
+    const int rc = launch_score_select(g, K, V, idx, score, ws, st, in_kernel);
     if (rc != LRSA_OK) return rc;
     woff += g.Wsel;
   }
@@ -207,6 +211,11 @@ const char* lrsa_status_string(int status) {
 }
 
 int lrsa_last_launch_count(void) { return launch_counter().n; }
+
+int lrsa_debug_set_wait_limit(int polls) {
+  set_unit_wait_limit(polls == 0 ? (1 << 21) : polls);
+  return LRSA_OK;
+}
 
 int lrsa_debug_set_impl(int impl) {
   if (impl != 0 && impl != 1) return LRSA_ERR_INVALID_ARG;

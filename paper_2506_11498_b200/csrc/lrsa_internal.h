@@ -74,7 +74,10 @@ int run_score_select(const lrsa_params_t* p, const Geom& whole, const __nv_bfloa
 // score_select.cu (one sequence; the status header of `ws` is cleared by the caller)
 size_t score_select_ws_bytes(const Geom& g);
 int launch_score_select(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat16* V, int32_t* idx,
-                        float* score, void* ws, cudaStream_t st);
+                        float* score, void* ws, cudaStream_t st, bool clear_status = false);
+// True when the kernel that scores `g` can clear the status word itself (clear_status above).
+bool score_select_clears_status(const Geom& g);
+void set_unit_wait_limit(int polls);
 
 // attn_ref.cu : CUDA-core reference kernels (one warp per row), used for validation.
 size_t attn_ref_fwd_ws_bytes(const Geom& g);

@@ -1,20 +1,27 @@
 // LagKV scoring and top-K selection (Section 3.2, Eq. 4-8 and the selection rule after Eq. 8).
 //
-// One launch streams K and V exactly once.  The work unit is a slice of TOK tokens of one lag
-// window of one (batch, KV head); a CTA takes units from a ticket counter in DESCENDING window
-// order and keeps its slice of K and V in registers for both phases:
-//   phase 1  per-channel min/max of the slice (packed bf16x2 compares, exact), folded into the
-//            window's statistics in global memory with order-preserving integer atomics, then
-//            a release-increment of the window's `ready` counter            (Eq. 4, Eq. 5)
-//   phase 2  wait (bounded) until the FOLLOWING window's statistics are complete, normalise
-//            the slice held in registers (Eq. 6), per-token standard deviation over head_dim
-//            (Eq. 7, inner part), written to a small fp32 scratch
-//   select   the CTA that finishes a window last soft-maxes the window's K and V spreads
-//            (Eq. 7), adds them (Eq. 8), radix-selects the top_k scores and emits the kept
-//            positions in ascending order.
-// A unit of window w waits only on units of window w+1, all of which hold smaller tickets, were
-// therefore picked up by CTAs that already run, and publish before they wait on anything: the
-// wait always ends, whatever the number of resident CTAs.  It is bounded all the same.
+// Two kernels, chosen by the lag window size:
+//   * score_select_chain_kernel (lag windows of up to 4096 tokens: the hot path).  A CTA owns a run of
+//     consecutive scored windows of one (batch, KV head), streams them downwards through a ring of bulk
+//     copies and keeps statistics and spreads in shared memory; no traffic between CTAs.  Described in
+//     front of the kernel below.
+//   * score_select_kernel (longer windows).  The work unit is a slice of TOK tokens of one lag window; a
+//     CTA takes one unit from a ticket counter in DESCENDING window order and keeps its slice of K and V
+//     in registers for both phases:
+//       phase 1  per-channel min/max of the slice (packed bf16x2 compares, exact), folded into the
+//                window's statistics in global memory with order-preserving integer atomics, then
+//                a release-increment of the window's `ready` counter            (Eq. 4, Eq. 5)
+//       phase 2  wait (bounded) until the FOLLOWING window's statistics are complete, normalise
+//                the slice held in registers (Eq. 6), per-token standard deviation over head_dim
+//                (Eq. 7, inner part), written to a small fp32 scratch
+//       select   the CTA that finishes a window last soft-maxes the window's K and V spreads
+//                (Eq. 7), adds them (Eq. 8), radix-selects the top_k scores and emits the kept
+//                positions in ascending order.
+//     A unit of window w waits only on units of window w+1, all of which hold smaller tickets, were
+//     therefore picked up by CTAs that already run, and publish before they wait on anything: the
+//     wait always ends, whatever the number of resident CTAs.  It is bounded all the same.
+// Both see one sequence: rows of N tokens per (batch, KV head), of which the sequence starts at token tok0
+// (packed batches), windows win_stride tokens apart (negative for the two-window ring of the inference cache).
 #include <stddef.h>
 
 #include "lrsa_internal.h"
@@ -42,6 +49,8 @@ struct ScoreArgs {
   int emit_off;           // added to S + w*L + i when a position is written to idx
   int win_stride;         // tokens from window w to window w+1 in memory (L; -L or L for a two-window ring buffer)
   long long elems;        // elements of K (and of V)
+  int clear_status;       // the chain kernel's first CTA clears the status word itself (saves a memset node)
+  int unit_wait_limit;    // polls of the one-slice-per-CTA kernel's wait for the next window; negative: give up at once
   int spin_limit;
 };
 
@@ -327,8 +336,8 @@ __global__ void __launch_bounds__(kThreads) score_select_kernel(const ScoreArgs 
   if (tid == 0) {
     const int* flag = a.ready + bh * a.W + w + 1;
     int it = 0;
-    while (ld_acquire(flag) < a.n_slices) {
-      if (++it > a.spin_limit) { s_flag = 1; atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT); break; }
+    while (a.unit_wait_limit < 0 || ld_acquire(flag) < a.n_slices) {
+      if (++it > a.unit_wait_limit) { s_flag = 1; atomicExch(&a.hdr->status, (int)LRSA_ERR_TIMEOUT); break; }
       __nanosleep(64);
     }
   }
@@ -419,10 +428,26 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
-__device__ __forceinline__ void group_sync(int grp) { asm volatile("bar.sync %0, 256;" ::"r"(grp + 1) : "memory"); }
 __device__ __forceinline__ void all_groups_sync() {
   asm volatile("bar.sync 3, %0;" ::"n"(kChainGroups * kThreads) : "memory");
 }
+// Barriers that also OR a predicate over their threads: every thread leaves with the same verdict, so a
+// group (or the whole CTA) takes the give-up branch together even if the flag was raised while some of
+// its threads had already looked at it.
+__device__ __forceinline__ bool bar_or(int id, int nthreads, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %3, 0;\n\t"
+      "bar.red.or.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(id), "r"(nthreads), "r"((uint32_t)pred)
+      : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ bool group_sync_or(int grp, bool pred) { return bar_or(grp + 1, kThreads, pred); }
+__device__ __forceinline__ bool all_groups_sync_or(bool pred) { return bar_or(3, kChainGroups * kThreads, pred); }
 
 // Bounded wait on a shared-memory barrier phase; false when it gave up.
 __device__ __forceinline__ bool stage_wait(uint32_t bar, uint32_t parity, int limit) {
@@ -451,6 +476,9 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
   __nv_bfloat16* red = reinterpret_cast<__nv_bfloat16*>(sel + select_scratch_bytes(a.L));   // [16 warps][4][D]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // A bounded wait needs seconds to expire, the first CTA of the grid starts with the launch: its clearing
+  // of the status word cannot overwrite another CTA's verdict.
+  if (a.clear_status && blockIdx.x == 0 && tid == 0) a.hdr->status = 0;
   if (tid == 0) {
     s_abort = 0;
     for (int i = 0; i < kChainGroups * kChainMaxRing; ++i) {
@@ -655,15 +683,14 @@ __global__ void __launch_bounds__(kChainThreads, 1) score_select_chain_kernel(co
       }
     }
     }
-    group_sync(grp);   // every read of the stage by this group is done
-    if (*abort) break;   // written before the barrier by whichever thread gave up
+    // every read of the stage by this group is done; one verdict for the group
+    if (group_sync_or(grp, *abort != 0)) break;
     if (gt == 0) ptx::mbar_arrive(ptx::smem_u32(&empty_bar[slot]));
     if (++ckr == ring) { ckr = 0; ++cuse; }
    }
 
    // ---- end of window w: both groups have written their spreads and hold their part of the statistics ----
-   all_groups_sync();
-   if (*abort) return;   // set before the barrier by whichever thread gave up
+   if (all_groups_sync_or(*abort != 0)) return;   // one verdict for the CTA
    if (scoring && grp == 0) select_window(a, bh, w, sel, true);   // group 0 only (its own barrier inside)
    if (want_stats) {
       // reduce the running statistics over the rows of a warp, then over the warps, and turn them
@@ -714,6 +741,11 @@ size_t select_smem_bytes(int L, int d) {
   return phase1 > sel ? phase1 : sel;
 }
 
+// Polls the one-slice-per-CTA kernel grants its wait for the following window's statistics.  Test hook:
+// a negative value makes that wait give up at once (the kernel holds its slice in registers and has no
+// copy in flight, so every thread returns after the verdict).  The chain kernel's limits are not touched.
+int g_unit_wait_limit = 1 << 21;
+
 struct ScoreWs {
   size_t ready, done, mm, zero_bytes, spread, total;
 };
@@ -736,8 +768,12 @@ ScoreWs score_ws_layout(const Geom& g) {
 // statistics and spreads.
 size_t score_select_ws_bytes(const Geom& g) { return g.L <= kChainMaxL ? sizeof(WsHeader) : score_ws_layout(g).total; }
 
+void set_unit_wait_limit(int polls) { g_unit_wait_limit = polls; }
+
+bool score_select_clears_status(const Geom& g) { return g.Wsel > 0 && g.L <= kChainMaxL; }
+
 int launch_score_select(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat16* V, int32_t* idx,
-                        float* score, void* ws, cudaStream_t st) {
+                        float* score, void* ws, cudaStream_t st, bool clear_status) {
   if (g.Wsel == 0) return LRSA_OK;  // nothing is scored
   const ScoreWs lay = score_ws_layout(g);
   unsigned char* base = static_cast<unsigned char*>(ws);
@@ -758,7 +794,9 @@ int launch_score_select(const Geom& g, const __nv_bfloat16* K, const __nv_bfloat
   a.tok0 = g.tok0; a.Wtot = g.Wtot; a.woff = g.woff; a.emit_off = g.emit_off; a.win_stride = g.win_stride;
   a.elems = (long long)g.B * g.Hkv * g.Nrow * g.d;
   a.ddof = g.ddof;
+  a.clear_status = clear_status && score_select_clears_status(g) ? 1 : 0;
   a.spin_limit = 1 << 21;
+  a.unit_wait_limit = g_unit_wait_limit;
   const int tok = g.d == 128 ? tok_per_unit<128>() : tok_per_unit<64>();
   a.n_slices = (g.L + tok - 1) / tok;
   const size_t smem = select_smem_bytes(g.L, g.d);

@@ -100,6 +100,8 @@ def lib() -> ctypes.CDLL:
         L.lrsa_status_string.restype = ctypes.c_char_p
         L.lrsa_last_launch_count.argtypes = []
         L.lrsa_debug_set_impl.argtypes = [ctypes.c_int]
+        L.lrsa_debug_set_wait_limit.argtypes = [ctypes.c_int]
+        L.lrsa_debug_set_wait_limit.restype = ctypes.c_int
         for name in ("lrsa_num_sel_windows", "lrsa_workspace_bytes", "lrsa_score_select", "lrsa_attn_fwd",
                      "lrsa_attn_bwd", "lrsa_workspace_status", "lrsa_last_launch_count", "lrsa_debug_set_impl"):
             getattr(L, name).restype = ctypes.c_int
@@ -217,6 +219,11 @@ def lrsa_workspace_status(workspace, stream=None) -> int:
 
 def lrsa_last_launch_count() -> int:
     return lib().lrsa_last_launch_count()
+
+
+def lrsa_debug_set_wait_limit(polls: int):
+    """Test hook: polls granted to the long-window scoring kernel's wait (negative: give up at once, 0: default)."""
+    _check(lib().lrsa_debug_set_wait_limit(int(polls)), "lrsa_debug_set_wait_limit")
 
 
 def lrsa_debug_set_impl(impl: int):

@@ -306,3 +306,25 @@ def test_query_chunk_of_several_lag_windows(m):
     for name, a, b, ref in zip(("dQ", "dK", "dV"), g1, gm, (odQ, odK, odV)):
         check_close(name, f64(b), ref)
         assert (a.float() - b.float()).abs().max().item() <= 2e-2
+
+
+def test_expired_wait_is_reported_and_the_next_call_is_clean():
+    """The bounded wait of the long-window scoring kernel, made to give up at once through the test hook:
+    the call returns, the workspace reports LRSA_ERR_TIMEOUT, and an ordinary call on the same workspace
+    afterwards is clean and correct."""
+    w = W("s_timeout", 1, 1, 1, 2 + 3 * 4608 + 11, 64, 4608, 100, 2, seed=42)
+    host = workloads.generate(w, ("K", "V"))
+    dev = to_dev(host)
+    p = lrsa.Params.from_workload(w)
+    ws = lrsa.new_workspace(lrsa.lrsa_workspace_bytes(p)[0])
+    want, _ = lrsa.lrsa_score_select(p, dev["K"], dev["V"], workspace=ws)
+    assert lrsa.lrsa_workspace_status(ws) == 0
+    lrsa.lrsa_debug_set_wait_limit(-1)
+    try:
+        lrsa.lrsa_score_select(p, dev["K"], dev["V"], workspace=ws)
+        assert lrsa.lrsa_workspace_status(ws) == 5      # LRSA_ERR_TIMEOUT
+    finally:
+        lrsa.lrsa_debug_set_wait_limit(0)
+    again, _ = lrsa.lrsa_score_select(p, dev["K"], dev["V"], workspace=ws)
+    assert lrsa.lrsa_workspace_status(ws) == 0
+    assert torch.equal(again, want)
