@@ -191,9 +191,10 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
-# DRAM bytes per backward call (dK/dV + dQ kernels) from the ncu summary under profiles/, per workload;
-# empty while the kernels are newer than the last capture (the record then carries null)
-BWD_DRAM_BYTES = {}
+# DRAM bytes per backward call (dK/dV + dQ kernels: dram__bytes_read.sum + dram__bytes_write.sum of one launch
+# each) from the ncu summary under profiles/, per workload; a workload without a capture of the current
+# kernels carries null
+BWD_DRAM_BYTES = {"cfg2_32k_gqa7_d128": 3.080e9}
 
 
 def spawn_ranks(n: int) -> int:
