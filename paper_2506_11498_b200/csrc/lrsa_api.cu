@@ -131,6 +131,7 @@ int lrsa_workspace_bytes(const lrsa_params_t* params, size_t* score_select, size
 
 int lrsa_score_select(const lrsa_params_t* params, const void* K, const void* V, int32_t* idx,
                       float* score, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  NvtxRange nvtx_range("lrsa_score_select");
   launch_counter().n = 0;
   Geom g;
   const int rc = make_geom(params, &g);
@@ -147,6 +148,7 @@ int lrsa_score_select(const lrsa_params_t* params, const void* K, const void* V,
 int lrsa_attn_fwd(const lrsa_params_t* params, const void* Q, const void* K, const void* V,
                   const int32_t* idx, void* O, float* LSE, void* workspace, size_t workspace_bytes,
                   void* cuda_stream) {
+  NvtxRange nvtx_range("lrsa_attn_fwd");
   launch_counter().n = 0;
   Geom g;
   const int rc = make_geom(params, &g);
@@ -167,6 +169,7 @@ int lrsa_attn_fwd(const lrsa_params_t* params, const void* Q, const void* K, con
 int lrsa_attn_bwd(const lrsa_params_t* params, const void* Q, const void* K, const void* V,
                   const void* O, const void* dO, const float* LSE, const int32_t* idx, void* dQ,
                   void* dK, void* dV, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  NvtxRange nvtx_range("lrsa_attn_bwd");
   launch_counter().n = 0;
   Geom g;
   const int rc = make_geom(params, &g);

@@ -313,6 +313,7 @@ int lrsa_cache_bytes(const lrsa_params_t* params, size_t* cache_bytes, size_t* w
 int lrsa_cache_append(const lrsa_params_t* params, void* cache, size_t cache_bytes, const void* k_new,
                       const void* v_new, int32_t n_prev, int32_t n_new, void* workspace, size_t workspace_bytes,
                       void* cuda_stream) {
+  NvtxRange nvtx_range("lrsa_cache_append");
   launch_counter().n = 0;
   Geom g;
   int rc = make_geom(params, &g);
@@ -390,6 +391,7 @@ int lrsa_cache_kept(const lrsa_params_t* params, const void* cache, const int32_
 int lrsa_attn_decode(const lrsa_params_t* params, const void* cache, size_t cache_bytes, const void* q,
                      int32_t n_tokens, void* o, float* lse, void* workspace, size_t workspace_bytes,
                      void* cuda_stream) {
+  NvtxRange nvtx_range("lrsa_attn_decode");
   launch_counter().n = 0;
   Geom g;
   const int rc = make_geom(params, &g);

@@ -6,6 +6,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/lrsa.h"
 
 namespace lrsa {
@@ -61,6 +63,14 @@ __host__ __device__ inline int first_compressed_chunk(int w, int ndp, int Wsel, 
   int c = w + 1 + ndp;
   return c < C ? c : C;
 }
+
+// NVTX range around an entry point (visible in a timeline profiler; free when no tool is attached).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+  NvtxRange(const NvtxRange&) = delete;
+  NvtxRange& operator=(const NvtxRange&) = delete;
+};
 
 struct LaunchCounter {
   int n = 0;

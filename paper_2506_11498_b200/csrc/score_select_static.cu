@@ -43,6 +43,7 @@ int static_scratch(void** out) {
 extern "C" int lrsa_score_select_static(const lrsa_params_t* params, const void* K, const void* V,
                                         int32_t* idx, float* score, void* cuda_stream) {
   using namespace lrsa;
+  NvtxRange nvtx_range("lrsa_score_select_static");
   launch_counter().n = 0;
   Geom g;
   const int rc = make_geom(params, &g);

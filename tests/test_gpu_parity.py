@@ -328,3 +328,45 @@ def test_expired_wait_is_reported_and_the_next_call_is_clean():
     again, _ = lrsa.lrsa_score_select(p, dev["K"], dev["V"], workspace=ws)
     assert lrsa.lrsa_workspace_status(ws) == 0
     assert torch.equal(again, want)
+
+
+def _padded(shape, dtype, fill, pad=4096):
+    """A tensor of `shape` carved out of a larger buffer whose margins hold a sentinel."""
+    n = int(np.prod(shape))
+    buf = torch.full((n + 2 * pad,), fill, dtype=dtype, device="cuda")
+    return buf, buf[pad:pad + n].view(shape)
+
+
+def _margins_intact(buf, n, fill, pad=4096):
+    ref = torch.full((pad,), fill, dtype=buf.dtype, device="cuda")
+    return torch.equal(buf[:pad], ref) and torch.equal(buf[pad + n:], ref)
+
+
+@pytest.mark.parametrize("w", [
+    W("canary_ragged", 1, 7, 1, 3 + 4 * 200 + 50, 128, 200, 50, 3, seed=61),      # nothing is a tile multiple
+    W("canary_d64", 2, 4, 2, 16 + 6 * 128 + 1, 64, 128, 32, 16, seed=62),
+], ids=lambda w: w.name)
+def test_outputs_never_written_outside_their_tensors(w):
+    """Every output tensor sits inside a larger buffer with sentinel margins: after the three calls the
+    margins are untouched (a stray store of a ragged tile, a bulk copy of a partial row or a reduction onto a
+    wrong row would show) and every element inside has been overwritten."""
+    host = workloads.generate(w)
+    dev = to_dev(host)
+    p = lrsa.Params.from_workload(w)
+    wsel = lrsa.lrsa_num_sel_windows(p)
+    bf, f32 = torch.bfloat16, torch.float32
+    bi, idx = _padded((w.B, w.Hkv, wsel, w.K), torch.int32, -7)
+    bs, sc = _padded((w.B, w.Hkv, wsel, w.L), f32, -7.0)
+    bO, O = _padded((w.B, w.Hq, w.N, w.d), bf, 777.0)
+    bL, LSE = _padded((w.B, w.Hq, w.N), f32, 777.0)
+    bQ, dQ = _padded((w.B, w.Hq, w.N, w.d), bf, 777.0)
+    bK, dK = _padded((w.B, w.Hkv, w.N, w.d), bf, 777.0)
+    bV, dV = _padded((w.B, w.Hkv, w.N, w.d), bf, 777.0)
+    lrsa.lrsa_score_select(p, dev["K"], dev["V"], idx=idx, score=sc)
+    lrsa.lrsa_attn_fwd(p, dev["Q"], dev["K"], dev["V"], idx, O=O, LSE=LSE)
+    lrsa.lrsa_attn_bwd(p, dev["Q"], dev["K"], dev["V"], O, dev["dO"], LSE, idx, dQ=dQ, dK=dK, dV=dV)
+    torch.cuda.synchronize()
+    for name, buf, t, fill in (("idx", bi, idx, -7), ("score", bs, sc, -7.0), ("O", bO, O, 777.0), ("LSE", bL, LSE, 777.0),
+                               ("dQ", bQ, dQ, 777.0), ("dK", bK, dK, 777.0), ("dV", bV, dV, 777.0)):
+        assert _margins_intact(buf, t.numel(), fill), f"{name}: a margin was written"
+        assert not (t == fill).any(), f"{name}: an element was left unwritten"
