@@ -93,7 +93,11 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // Top-K of the window by the last CTA to finish it.  smem: sk[L], sv[L] floats, then scratch.
 // Bytes of the selection scratch: sk[L], sv[L], 256 histogram bins, 32 floats, 16 ints.
-__host__ __device__ inline size_t select_scratch_bytes(int L) { return (size_t)2 * L * 4 + 256 * 4 + 32 * 4 + 16 * 4; }
+// Rounded up to 16 bytes: the chain kernel puts a buffer of 16-byte vectors right behind this scratch
+// (an odd window length would leave it misaligned otherwise).
+__host__ __device__ inline size_t select_scratch_bytes(int L) {
+  return (((size_t)2 * L * 4 + 256 * 4 + 32 * 4 + 16 * 4) + 15) & ~(size_t)15;
+}
 
 // Barrier of the 256 scoring threads (named barrier 1): the whole block in the one-unit-per-CTA kernel,
 // all warps but the producer in the streaming kernel.

@@ -44,7 +44,7 @@ def error_stats(got, want):
             "n": int(err.size)}
 
 
-def check_close(name, got, want, max_abs=MAX_ABS, rel_l2=REL_L2, ulp=BF16_ULP, terms=None):
+def check_close(name, got, want, max_abs=MAX_ABS, rel_l2=REL_L2, ulp=BF16_ULP, terms=None, extra=None):
     """Element-wise |got - want| <= max_abs + ulp * |want| and relative L2 <= rel_l2.  Prints and
     records the unscaled maximum error next to the verdict.  `terms` (same shape, optional): the sum of
     the absolute terms that make up each element; ulp * terms is added to the bound (forward error of a
@@ -61,6 +61,8 @@ def check_close(name, got, want, max_abs=MAX_ABS, rel_l2=REL_L2, ulp=BF16_ULP, t
     bound = max_abs + ulp * np.abs(want)
     if terms is not None:
         bound = bound + ulp * np.asarray(terms, np.float64)
+    if extra is not None:          # an absolute allowance per element, derived by the caller
+        bound = bound + np.asarray(extra, np.float64)
     worst = int(np.argmax(err - bound))
     assert (err <= bound).all(), f"{name}: |err|={err.flat[worst]:.4g} at {worst} (ref {want.flat[worst]:.4g})"
     assert st["rel_l2"] <= rel_l2, f"{name}: relative L2 {st['rel_l2']:.3g} > {rel_l2}"
@@ -99,3 +101,40 @@ def to_dev(host):
 
 def f64(t):
     return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def gradient_error_terms(w, op, bits, oidx, oO, oL, cu=()):
+    """Quantities, from the oracle's values (numpy, fp64, dense [N,N] per head: small cases only), that
+    bound what the arithmetic of a bf16 tensor-core backward can do to a gradient element:
+      mQ, mK, mV : sums of the absolute terms of each element of dQ, dK, dV
+                     dQ[t,c] = scale * sum_j dS[t,j] K[j,c]  ->  scale * sum_j |dS[t,j]| |K[j,c]|   (dK alike with Q)
+                     dV[j,c] = sum_t P[t,j] dO[t,c]           ->  sum_t P[t,j] |dO[t,c]|
+                   a product whose left operand is rounded to bf16 (P and dS are, to reach the tensor
+                   cores) errs by up to 2^-9 of that sum, however small the cancelled result is;
+      dK_from_D  : what the rounding of O to bf16 does to dK through D = rowsum(dO * O), which the dK/dV
+                   kernel takes from the stored O: delta_t (four standard deviations of a sum of d
+                   independent roundings of relative size 2^-9) enters dS[t,j] as P[t,j] * delta_t, hence
+                   dK[j,c] as scale * sum_t P[t,j] |delta_t| |Q[t,c]|.  It matters where a query puts most
+                   of its weight on one key (the first tokens of a sequence, dominant keys)."""
+    G = w.Hq // w.Hkv
+    scale = 1.0 / np.sqrt(w.d)
+    Q, K, V, dO = (orc.bits_to_f64(bits[k]) for k in ("Q", "K", "V", "dO"))
+    mQ, mK, mV, tK = np.zeros_like(Q), np.zeros_like(K), np.zeros_like(V), np.zeros_like(K)
+    for b in range(w.B):
+        for hq in range(w.Hq):
+            h = hq // G
+            if cu:
+                vis = np.stack([orc.visible_row_packed(op, oidx, cu, b, h, t) for t in range(w.N)])
+            else:
+                vis = np.stack([orc.visible_row(op, oidx, b, h, t) for t in range(w.N)])
+            S = (Q[b, hq] @ K[b, h].T) * scale
+            P = np.where(vis, np.exp(S - oL[b, hq][:, None]), 0.0)
+            dP = dO[b, hq] @ V[b, h].T
+            D = (P * dP).sum(-1, keepdims=True)
+            dS = np.abs(P * (dP - D))
+            mQ[b, hq] = scale * dS @ np.abs(K[b, h])
+            mK[b, h] += scale * dS.T @ np.abs(Q[b, hq])
+            mV[b, h] += P.T @ np.abs(dO[b, hq])
+            delta = 4.0 * 2.0 ** -9 / np.sqrt(3.0) * np.sqrt(((dO[b, hq] * oO[b, hq]) ** 2).sum(-1, keepdims=True))
+            tK[b, h] += scale * P.T @ (delta * np.abs(Q[b, hq]))
+    return {"mQ": mQ, "mK": mK, "mV": mV, "dK_from_D": tK}

@@ -7,7 +7,7 @@ import torch
 
 from oracle import lrsa_oracle as orc
 from paper_2506_11498_b200 import lrsa, workloads
-from tests.parity_utils import (REPORT, check_close, compare_idx, error_stats, f64, host_bits, oparams, to_dev)
+from tests.parity_utils import (REPORT, check_close, gradient_error_terms, compare_idx, error_stats, f64, host_bits, oparams, to_dev)
 
 pytestmark = pytest.mark.gpu
 
@@ -99,31 +99,6 @@ def _run_attention(w, ndp, idx_np, host, impl=0):
     return O, LSE, dQ, dK, dV
 
 
-def _term_magnitudes(w, op, bits, oidx, oL):
-    """Sums of the absolute terms of every gradient element, from the oracle's quantities (numpy, fp64):
-       dQ[t,c] = scale * sum_j dS[t,j] K[j,c]   ->  scale * sum_j |dS[t,j]| |K[j,c]|     (same for dK with Q)
-       dV[j,c] = sum_t P[t,j] dO[t,c]           ->  sum_t P[t,j] |dO[t,c]|
-    A product whose left operand is rounded to bf16 (P and dS are, to reach the tensor cores) errs by up
-    to 2^-9 of this sum, however small the cancelled result is."""
-    G = w.Hq // w.Hkv
-    scale = 1.0 / np.sqrt(w.d)
-    Q, K, V, dO = (orc.bits_to_f64(bits[k]) for k in ("Q", "K", "V", "dO"))
-    mQ, mK, mV = np.zeros_like(Q), np.zeros_like(K), np.zeros_like(V)
-    for b in range(w.B):
-        for hq in range(w.Hq):
-            h = hq // G
-            vis = np.stack([orc.visible_row(op, oidx, b, h, t) for t in range(w.N)])
-            S = (Q[b, hq] @ K[b, h].T) * scale
-            P = np.where(vis, np.exp(S - oL[b, hq][:, None]), 0.0)
-            dP = dO[b, hq] @ V[b, h].T
-            D = (P * dP).sum(-1, keepdims=True)
-            dS = np.abs(P * (dP - D))
-            mQ[b, hq] = scale * dS @ np.abs(K[b, h])
-            mK[b, h] += scale * dS.T @ np.abs(Q[b, hq])
-            mV[b, h] += P.T @ np.abs(dO[b, hq])
-    return mQ, mK, mV
-
-
 @pytest.mark.parametrize("w,ndp", ATTN_CASES, ids=lambda x: x.name if hasattr(x, "name") else str(x))
 def test_attention_fwd_bwd(w, ndp):
     host = workloads.generate(w)
@@ -138,10 +113,10 @@ def test_attention_fwd_bwd(w, ndp):
     if w.values == "salient":
         # The deliberately ill-conditioned case (700 tokens, d = 64, a handful of keys scaled by 8): its
         # gradient elements are cancelling sums of large terms, and the bound follows the terms.
-        mQ, mK, mV = _term_magnitudes(w, op, bits, oidx, oL)
-        check_close("dQ", f64(dQ), odQ, terms=mQ)
-        check_close("dK", f64(dK), odK, terms=mK)
-        check_close("dV", f64(dV), odV, terms=mV)
+        e = gradient_error_terms(w, op, bits, oidx, oO, oL)
+        check_close("dQ", f64(dQ), odQ, terms=e["mQ"])
+        check_close("dK", f64(dK), odK, terms=e["mK"], extra=e["dK_from_D"])
+        check_close("dV", f64(dV), odV, terms=e["mV"])
     else:
         check_close("dQ", f64(dQ), odQ)
         check_close("dK", f64(dK), odK)
