@@ -74,6 +74,13 @@ typedef struct lrsa_params {
                             token axis of every batch element holds n_seqs sequences back to back */
   const int32_t* cu_seqlens; /* HOST pointer, n_seqs + 1 boundaries: cu_seqlens[0] = 0, increasing,
                             cu_seqlens[n_seqs] = seq_len.  Read during the call only.  NULL when n_seqs = 0 */
+  void* o_residual;      /* optional DEVICE pointer, bf16 [B, Hq, N, d], 16-byte aligned, or NULL.  The paper has no
+                            counterpart: it is the part of the attention output that the bf16 O cannot hold.
+                            lrsa_attn_fwd writes bf16(O_fp32 - O) there; lrsa_attn_bwd, given the buffer the
+                            forward of the same inputs filled, takes the D = rowsum(dO * O) that dK is formed
+                            with over O + o_residual.  That removes the rounding of O from dK (it matters where
+                            a query puts nearly all its weight on one key); dQ does not depend on it (its D is
+                            the exact sum_j P dP) and dV has no D.  The other calls ignore the field. */
 } lrsa_params_t;
 
 /* Number of scored windows W_sel (see Geometry).  idx has W_sel * top_k entries per KV head. */

@@ -320,36 +320,41 @@ lrsa_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
 
 // Per query row: D~_t = sum_c dO[t,c] * O[t,c] and -LSE_t * log2(e).  d/8 lanes share a row (16 bytes
 // each) and a warp takes kPrepUnroll groups of 256/d rows with all loads issued before the arithmetic:
-// the kernel only streams O and dO once and should run at memory speed.
+// the kernel only streams O and dO once and should run at memory speed.  With the rounding remainder of O
+// (Olo, optional) the sum runs over O + Olo, which is O to fp32 accuracy.
 constexpr int kPrepUnroll = 4;
-__global__ void bwd_prep_kernel(const __nv_bfloat16* __restrict__ O, const __nv_bfloat16* __restrict__ dO,
-                                const float* __restrict__ LSE, float2* __restrict__ stats, long long rows, int d) {
+__global__ void bwd_prep_kernel(const __nv_bfloat16* __restrict__ O, const __nv_bfloat16* __restrict__ Olo,
+                                const __nv_bfloat16* __restrict__ dO, const float* __restrict__ LSE,
+                                float2* __restrict__ stats, long long rows, int d) {
   const int lane = threadIdx.x & 31;
   const int lpr = d >> 3, rpw = 32 / lpr;   // lanes per row, rows per warp-wide load (d = 64: 8, 4; d = 128: 16, 2)
   const long long warp_id = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const long long row0 = warp_id * (kPrepUnroll * rpw) + lane / lpr;
   const int c = (lane % lpr) * 8;
-  uint4 o[kPrepUnroll], g[kPrepUnroll];
+  uint4 o[kPrepUnroll], l[kPrepUnroll], g[kPrepUnroll];
 #pragma unroll
   for (int u = 0; u < kPrepUnroll; ++u) {
     const long long row = row0 + u * rpw;
+    o[u] = l[u] = g[u] = make_uint4(0, 0, 0, 0);
     if (row < rows) {
       o[u] = *reinterpret_cast<const uint4*>(O + row * d + c);
       g[u] = *reinterpret_cast<const uint4*>(dO + row * d + c);
-    } else {
-      o[u] = make_uint4(0, 0, 0, 0);
-      g[u] = make_uint4(0, 0, 0, 0);
+      if (Olo) l[u] = *reinterpret_cast<const uint4*>(Olo + row * d + c);
     }
   }
 #pragma unroll
   for (int u = 0; u < kPrepUnroll; ++u) {
     const uint32_t ow[4] = {o[u].x, o[u].y, o[u].z, o[u].w}, gw[4] = {g[u].x, g[u].y, g[u].z, g[u].w};
-    float acc = 0.f;
+    const uint32_t lw[4] = {l[u].x, l[u].y, l[u].z, l[u].w};
+    float acc = 0.f, acc_lo = 0.f;   // the remainder's products are 2^-9 of the others: summed apart, added last
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       acc = fmaf(__uint_as_float(ow[j] << 16), __uint_as_float(gw[j] << 16), acc);
       acc = fmaf(__uint_as_float(ow[j] & 0xffff0000u), __uint_as_float(gw[j] & 0xffff0000u), acc);
+      acc_lo = fmaf(__uint_as_float(lw[j] << 16), __uint_as_float(gw[j] << 16), acc_lo);
+      acc_lo = fmaf(__uint_as_float(lw[j] & 0xffff0000u), __uint_as_float(gw[j] & 0xffff0000u), acc_lo);
     }
+    acc += acc_lo;
     for (int off = lpr >> 1; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
     const long long row = row0 + u * rpw;
     if ((lane % lpr) == 0 && row < rows) stats[row] = make_float2(-LSE[row] * 1.4426950408889634f, acc);
@@ -389,11 +394,11 @@ __global__ void __launch_bounds__(256) kbar_kernel(const __nv_bfloat16* __restri
 
 }  // namespace
 
-int launch_bwd_prep(const Geom& g, const __nv_bfloat16* O, const __nv_bfloat16* dO, const float* LSE,
-                    const __nv_bfloat16* K, float2* stats, float* kbar, cudaStream_t st) {
+int launch_bwd_prep(const Geom& g, const __nv_bfloat16* O, const __nv_bfloat16* Olo, const __nv_bfloat16* dO,
+                    const float* LSE, const __nv_bfloat16* K, float2* stats, float* kbar, cudaStream_t st) {
   const long long rows = (long long)g.B * g.Hq * g.N;
   const long long rows_per_block = 8LL * kPrepUnroll * (32 / (g.d >> 3));
-  bwd_prep_kernel<<<(unsigned)((rows + rows_per_block - 1) / rows_per_block), 256, 0, st>>>(O, dO, LSE, stats, rows, g.d);
+  bwd_prep_kernel<<<(unsigned)((rows + rows_per_block - 1) / rows_per_block), 256, 0, st>>>(O, Olo, dO, LSE, stats, rows, g.d);
   LRSA_CUDA_CHECK(cudaGetLastError());
   launch_counter().n++;
   const int nsplit = 64, rpb = (g.N + nsplit - 1) / nsplit;

@@ -45,7 +45,8 @@ int launch_attn_bwd_sm100(const lrsa_params_t* params, const Geom& g, const __nv
   // Per-row statistics and the mean key are taken over whole rows (the mean key is only a centring
   // vector: any constant works).  Then, sequence after sequence, the dK/dV kernel (which also produces
   // the accurate D of the sequence's rows) and the dQ kernel; bf16 dK, dV at the end.
-  int rc = launch_bwd_prep(g, O, dO, LSE, K, stats, kbar, st);
+  const __nv_bfloat16* Olo = static_cast<const __nv_bfloat16*>(params->o_residual);
+  int rc = launch_bwd_prep(g, O, Olo, dO, LSE, K, stats, kbar, st);
   if (rc == LRSA_OK) rc = dkv_zero(g, base + lay.dkv, st);
   const int n_seqs = geom_n_seqs(params);
   int woff = 0;

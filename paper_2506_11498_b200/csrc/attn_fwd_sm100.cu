@@ -37,6 +37,7 @@ struct FwdArgs {
   BlockPlan plan;
   int BH, Hq, Hkv, G, N;   // N: tokens per (batch, head) row of O and LSE (the row stride)
   __nv_bfloat16* O;
+  __nv_bfloat16* Olo;        // optional: receives bf16(O_fp32 - O), the part of the output the bf16 O cannot hold
   float* LSE;
   float scale, scale_log2;   // softmax scale, and scale * log2(e)
   int* status;
@@ -313,6 +314,8 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       const float lt = red_s[0][row] + red_s[1][row];
       const float inv = 1.0f / lt;
       unsigned char* srow = stage_out + row * kStageStride + half * (kRowBytes / 2);
+      // the remainder goes straight to global memory (64 or 128 contiguous bytes per thread, written once)
+      __nv_bfloat16* lo_row = a.Olo && store ? a.Olo + ((size_t)bh * a.N + qpos) * D + half * (D / 2) : nullptr;
 #pragma unroll
       for (int q = 0; q < D / 64; ++q) {
         uint32_t o[32];
@@ -320,12 +323,21 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         tmem_wait_ld();
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
+          float f[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(o[8 * v + e]) * inv;
           uint4 w;
-          w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
-          w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
-          w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
-          w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+          w.x = pack_bf16(f[0], f[1]); w.y = pack_bf16(f[2], f[3]);
+          w.z = pack_bf16(f[4], f[5]); w.w = pack_bf16(f[6], f[7]);
           *reinterpret_cast<uint4*>(srow + (q * 4 + v) * 16) = w;
+          if (lo_row) {
+            const uint32_t hw[4] = {w.x, w.y, w.z, w.w};
+            uint32_t lw[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              lw[e] = pack_bf16(f[2 * e] - __uint_as_float(hw[e] << 16), f[2 * e + 1] - __uint_as_float(hw[e] & 0xffff0000u));
+            *reinterpret_cast<uint4*>(lo_row + q * 32 + v * 8) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+          }
         }
       }
       if (store && half == 0) a.LSE[(size_t)bh * a.N + qpos] = m * a.scale + logf(lt);
@@ -442,8 +454,8 @@ size_t attn_fwd_ws_bytes(const Geom& g) { return fwd_ws_layout(g).total; }
 
 template <int D>
 static int launch_fwd_t(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* K, const __nv_bfloat16* V,
-                        const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, __nv_bfloat16* O, float* LSE, int* status,
-                        cudaStream_t st) {
+                        const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, __nv_bfloat16* O, __nv_bfloat16* Olo, float* LSE,
+                        int* status, cudaStream_t st) {
   using Cfg = FwdCfg<D>;
   CUtensorMap mQ, mK, mV, mKc, mVc;
   const long long rc = g.Rc > 0 ? g.Rc : 1;
@@ -458,7 +470,7 @@ static int launch_fwd_t(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat
   FwdArgs a;
   a.plan = make_plan(g, kTile);
   a.BH = g.B * g.Hq; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.N = g.Nrow;
-  a.O = O + sh; a.LSE = LSE + g.tok0; a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f;
+  a.O = O + sh; a.Olo = Olo ? Olo + sh : nullptr; a.LSE = LSE + g.tok0; a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f;
   a.status = status;
   const long long grid = (long long)a.plan.total * a.BH;
   if (grid > 0x7fffffffLL) return LRSA_ERR_UNSUPPORTED;
@@ -481,6 +493,7 @@ int launch_attn_fwd_sm100(const lrsa_params_t* params, const Geom& g, const __nv
   __nv_bfloat16* Kc = reinterpret_cast<__nv_bfloat16*>(base + lay.kc);
   __nv_bfloat16* Vc = reinterpret_cast<__nv_bfloat16*>(base + lay.vc);
   int* status = &reinterpret_cast<WsHeader*>(base)->status;
+  __nv_bfloat16* Olo = static_cast<__nv_bfloat16*>(params->o_residual);
   // sequence after sequence (one for an unpacked batch); the compact buffers are reused in stream order
   const int n_seqs = geom_n_seqs(params);
   int woff = 0;
@@ -490,8 +503,8 @@ int launch_attn_fwd_sm100(const lrsa_params_t* params, const Geom& g, const __nv
     woff += gs.Wsel;
     int rc = launch_compact_kv(gs, K, V, idx, Kc, Vc, st);
     if (rc == LRSA_OK)
-      rc = gs.d == 128 ? launch_fwd_t<128>(gs, Q, K, V, Kc, Vc, O, LSE, status, st)
-                       : launch_fwd_t<64>(gs, Q, K, V, Kc, Vc, O, LSE, status, st);
+      rc = gs.d == 128 ? launch_fwd_t<128>(gs, Q, K, V, Kc, Vc, O, Olo, LSE, status, st)
+                       : launch_fwd_t<64>(gs, Q, K, V, Kc, Vc, O, Olo, LSE, status, st);
     if (rc != LRSA_OK) return rc;
   }
   return LRSA_OK;

@@ -39,6 +39,8 @@ int make_geom(const lrsa_params_t* p, Geom* g) {
   g->Wsel = g->W > 1 ? g->W - 1 : 0;
   g->Rc = g->S + g->Wsel * g->K;
   g->Nrow = g->N; g->tok0 = 0; g->Wtot = g->Wsel; g->woff = 0; g->emit_off = 0; g->win_stride = g->L;
+  if (reinterpret_cast<uintptr_t>(p->o_residual) & 15u) return LRSA_ERR_INVALID_ARG;
+  g->has_o_res = p->o_residual != nullptr;
   if (p->n_seqs < 0) return LRSA_ERR_INVALID_ARG;
   if (p->n_seqs > 0) {
     if (!p->cu_seqlens || p->cu_seqlens[0] != 0 || p->cu_seqlens[p->n_seqs] != p->seq_len) return LRSA_ERR_INVALID_ARG;

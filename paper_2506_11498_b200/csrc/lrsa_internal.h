@@ -30,6 +30,7 @@ struct Geom {
   // Scoring only: value added to the positions written to idx (tok0 unless the rows are a ring buffer)
   // and distance in tokens from window w to window w+1 (L unless the rows are a ring buffer).
   int emit_off, win_stride;
+  int has_o_res;   // the caller gave a buffer for the rounding remainder of O (lrsa_params_t::o_residual)
 };
 
 // Sequence s of a packed batch (cu = boundaries, n_seqs + 1 entries) as a Geom of its own.
@@ -120,8 +121,8 @@ int launch_attn_bwd_sm100(const lrsa_params_t* params, const Geom& g, const __nv
 // Backward helpers.  stats[row] = (-LSE * log2(e), rowsum(dO * O)) per query row; kbar[b*Hkv+h][c] is the
 // mean key (accumulated into a zeroed array).  The dK/dV kernel runs first and adds sum_j P dP, the
 // accurate D of every query row, into the zeroed Dacc; the dQ kernel reads it.
-int launch_bwd_prep(const Geom& g, const __nv_bfloat16* O, const __nv_bfloat16* dO, const float* LSE,
-                    const __nv_bfloat16* K, float2* stats, float* kbar, cudaStream_t st);
+int launch_bwd_prep(const Geom& g, const __nv_bfloat16* O, const __nv_bfloat16* Olo, const __nv_bfloat16* dO,
+                    const float* LSE, const __nv_bfloat16* K, float2* stats, float* kbar, cudaStream_t st);
 int launch_bwd_dq_sm100(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat16* dO, const __nv_bfloat16* K,
                         const __nv_bfloat16* V, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc, const float2* stats,
                         const float* Dacc, const float* kbar, __nv_bfloat16* dQ, int* status, cudaStream_t st);

@@ -30,7 +30,8 @@ class lrsa_params_t(ctypes.Structure):
                 ("batch", "n_q_heads", "n_kv_heads", "seq_len", "head_dim", "chunk", "lag", "top_k",
                  "n_sink", "n_dense_prev", "std_ddof")] + [("softmax_scale", ctypes.c_float),
                                                            ("n_seqs", ctypes.c_int32),
-                                                           ("cu_seqlens", ctypes.POINTER(ctypes.c_int32))]
+                                                           ("cu_seqlens", ctypes.POINTER(ctypes.c_int32)),
+                                                           ("o_residual", ctypes.c_void_p)]
 
 
 @dataclass(frozen=True)
@@ -50,10 +51,12 @@ class Params:
     softmax_scale: float = 0.0
     cu_seqlens: tuple = ()    # packed batch: boundaries (0, ..., seq_len) of the sequences on the token axis
 
-    def c(self) -> lrsa_params_t:
+    def c(self, o_residual=None) -> lrsa_params_t:
+        """The C struct; `o_residual`: a bf16 tensor shaped like O (or None), see lrsa_attn_fwd."""
         cp = lrsa_params_t(self.batch, self.n_q_heads, self.n_kv_heads, self.seq_len, self.head_dim,
                            self.chunk or self.lag, self.lag, self.top_k, self.n_sink,
-                           self.n_dense_prev, self.std_ddof, self.softmax_scale, 0, None)
+                           self.n_dense_prev, self.std_ddof, self.softmax_scale, 0, None,
+                           None if o_residual is None else o_residual.data_ptr())
         if self.cu_seqlens:
             arr = (ctypes.c_int32 * len(self.cu_seqlens))(*self.cu_seqlens)
             cp.n_seqs = len(self.cu_seqlens) - 1
@@ -182,22 +185,23 @@ def lrsa_score_select_static_status(stream=None) -> int:
     return lib().lrsa_score_select_static_status(_stream(stream))
 
 
-def lrsa_attn_fwd(params: Params, Q, K, V, idx, O=None, LSE=None, workspace=None, stream=None):
-    """Eq. 3 under the chunked mask.  Returns (O bf16 [B,Hq,N,d], LSE fp32 [B,Hq,N])."""
+def lrsa_attn_fwd(params: Params, Q, K, V, idx, O=None, LSE=None, workspace=None, stream=None, o_residual=None):
+    """Eq. 3 under the chunked mask.  Returns (O bf16 [B,Hq,N,d], LSE fp32 [B,Hq,N]).  `o_residual` (bf16,
+    shaped like O, optional) receives what the bf16 O cannot hold; lrsa_attn_bwd takes it to form dK more accurately."""
     if O is None:
         O = torch.empty_like(Q)
     if LSE is None:
         LSE = torch.empty(Q.shape[:3], dtype=torch.float32, device=Q.device)
     if workspace is None:
         workspace = new_workspace(lrsa_workspace_bytes(params)[1], Q.device)
-    cp = params.c()
+    cp = params.c(o_residual)
     _check(lib().lrsa_attn_fwd(ctypes.byref(cp), _p(Q), _p(K), _p(V), _p(idx), _p(O), _p(LSE), _p(workspace),
                                workspace.numel(), _stream(stream)), "lrsa_attn_fwd")
     return O, LSE
 
 
 def lrsa_attn_bwd(params: Params, Q, K, V, O, dO, LSE, idx, dQ=None, dK=None, dV=None, workspace=None,
-                  stream=None):
+                  stream=None, o_residual=None):
     """Gradient of Eq. 3 with the mask constant.  Returns (dQ, dK, dV) in bf16."""
     if dQ is None:
         dQ = torch.empty_like(Q)
@@ -207,7 +211,7 @@ def lrsa_attn_bwd(params: Params, Q, K, V, O, dO, LSE, idx, dQ=None, dK=None, dV
         dV = torch.empty_like(V)
     if workspace is None:
         workspace = new_workspace(lrsa_workspace_bytes(params)[2], Q.device)
-    cp = params.c()
+    cp = params.c(o_residual)
     _check(lib().lrsa_attn_bwd(ctypes.byref(cp), _p(Q), _p(K), _p(V), _p(O), _p(dO), _p(LSE), _p(idx), _p(dQ),
                                _p(dK), _p(dV), _p(workspace), workspace.numel(), _stream(stream)), "lrsa_attn_bwd")
     return dQ, dK, dV

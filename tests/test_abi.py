@@ -90,3 +90,13 @@ def test_packed_parameter_validation():
             lrsa.lrsa_num_sel_windows(lrsa.Params(**GOOD, cu_seqlens=bad))
         assert e.value.status == 1
     assert lrsa.lrsa_num_sel_windows(lrsa.Params(**{**GOOD, "chunk": 256})) == (1000 - 4) // 128 - 1
+
+
+def test_o_residual_must_be_16_byte_aligned():
+    import ctypes
+    out = ctypes.c_int32(0)
+    cp = lrsa.Params(**GOOD).c()
+    cp.o_residual = 4096
+    assert lrsa.lib().lrsa_num_sel_windows(ctypes.byref(cp), ctypes.byref(out)) == 0
+    cp.o_residual = 4096 + 8
+    assert lrsa.lib().lrsa_num_sel_windows(ctypes.byref(cp), ctypes.byref(out)) == 1

@@ -77,6 +77,21 @@ def test_random_geometry(seed):
     # gradient_error_terms, measured at 2.2e-2 on one element of these cases)
     check_close("dK", f64(dK), odK, extra=gradient_error_terms(w, op, bits, oidx, oO, oL, cu)["dK_from_D"])
     check_close("dV", f64(dV), odV)
+    # with the rounding remainder of O: same O and LSE, the remainder is what the bf16 O lacks, and dK needs
+    # no allowance
+    R = torch.full_like(O, float("nan"))
+    ws2 = lrsa.new_workspace(lrsa.lrsa_workspace_bytes(p)[2])
+    O2, LSE2 = lrsa.lrsa_attn_fwd(p, dev["Q"], dev["K"], dev["V"], gi, workspace=ws[1], o_residual=R)
+    assert torch.equal(O2, O) and torch.equal(LSE2, LSE)
+    assert torch.isfinite(R.float()).all()
+    assert (R.float().abs() <= O.float().abs() * 2.0 ** -8 + 1e-30).all()
+    check_close("O + residual", f64(O) + f64(R), oO)
+    dQ2, dK2, dV2 = lrsa.lrsa_attn_bwd(p, dev["Q"], dev["K"], dev["V"], O, dev["dO"], LSE, gi, workspace=ws2,
+                                       o_residual=R)
+    assert lrsa.lrsa_workspace_status(ws2) == 0
+    check_close("dQ (residual)", f64(dQ2), odQ)
+    check_close("dK (residual)", f64(dK2), odK)
+    check_close("dV (residual)", f64(dV2), odV)
 
 
 @pytest.mark.parametrize("seed", range(100, 110))
