@@ -188,7 +188,8 @@ int lrsa_attn_bwd(const lrsa_params_t* params, const void* Q, const void* K, con
  *   k_new, v_new in : bf16 [B, Hkv, n_new, d]
  *
  * lrsa_attn_decode: Eq. 3 for ONE query token per (batch, query head), the token at position n_tokens - 1 of a
- * cache that holds n_tokens tokens; it sees exactly what row n_tokens - 1 of lrsa_attn_fwd sees.  fp32 arithmetic.
+ * cache that holds n_tokens tokens; it sees exactly what row n_tokens - 1 of lrsa_attn_fwd sees.  bf16 tensor-core products,
+ * fp32 accumulation and softmax, as in lrsa_attn_fwd.
  *   q in : bf16 [B, Hq, d];  o out : bf16 [B, Hq, d];  lse out (optional) : fp32 [B, Hq]
  *
  * lrsa_cache_kept returns a device pointer into the cache: int32 [B, Hkv, w_cap, top_k], the kept positions of the

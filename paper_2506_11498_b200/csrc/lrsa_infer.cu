@@ -88,8 +88,8 @@ __global__ void cache_keep_kernel(const int32_t* __restrict__ idx, const __nv_bf
 
 // ---- decode attention ----
 constexpr int kDecThreads = 128;
-constexpr int kDecHeads = 8;      // query heads of a group handled per pass over the keys
-constexpr int kDecKeys = 128;     // keys per CTA, staged in shared memory by bulk copies
+constexpr int kDecHeads = 16;     // query heads of a group per pass over the keys (the M of the tensor-core product)
+constexpr int kDecKeys = 128;     // keys per CTA (32 per warp), staged in shared memory
 
 struct DecodeArgs {
   const __nv_bfloat16 *q, *k_list, *v_list, *k_ring, *v_ring;
@@ -101,151 +101,196 @@ struct DecodeArgs {
   float scale_log2;
 };
 
-__device__ __forceinline__ float bf_lo(uint32_t p) { return __uint_as_float(p << 16); }
-__device__ __forceinline__ float bf_hi(uint32_t p) { return __uint_as_float(p & 0xffff0000u); }
-
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col)
+__device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// Grid (n_split, BHkv).  The CTA's (at most) 128 keys are runs of consecutive rows of the list and of the
-// ring (at most three runs: the ring wraps once); one thread fetches K and V of every run with bulk copies,
-// so all of the CTA's bytes are in flight at once.  Then D/8 lanes share a key (16 bytes each), a warp works
-// on 32/(D/8) keys at a time, and every such lane group keeps an online softmax (maximum, sum, 8 output
-// channels per lane) per query head.
+// Grid (n_split, BHkv).  One query token per (batch, head) and a few hundred to a few thousand keys per KV head:
+// the work is the transfer of K and V, so the CTA's (at most) 128 key rows are fetched by all threads at once
+// (one row of K and of V per thread, 16-byte asynchronous copies) and everything after that has to be short.
+// The query heads of the KV group form the rows of a small matrix product (GQA: 16 rows per pass, the unused
+// ones zero), so S = Q K^T and O = P V run on the warp-level tensor-core instructions (m16n8k16, bf16 operands,
+// fp32 accumulation; a 128-row tcgen05 product would be nine tenths padding here): a warp takes 32 keys, holds
+// Q as A fragments, reads K and V fragments with ldmatrix from rows whose 16-byte chunks are XOR-swizzled by the
+// row number (rows are 128 or 256 bytes apart, eight rows of one chunk would share their banks), forms the
+// softmax of its 32 keys in registers and hands P over as the A operand of the second product.  The four
+// warps' partial results are merged through shared memory; the splits by decode_merge_kernel.
 template <int D>
 __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const DecodeArgs a) {
-  constexpr int LPK = D / 8, KPW = 32 / LPK;           // lanes per key, keys per warp step
-  constexpr int kGroups = (kDecThreads / 32) * KPW;    // lane groups per CTA
-  extern __shared__ __align__(128) unsigned char dec_smem[];   // K rows [kDecKeys][D], then V rows
-  __shared__ __align__(8) uint64_t bar;
-  __shared__ float red_m[kGroups][kDecHeads], red_l[kGroups][kDecHeads];
-  __shared__ float red_o[kGroups][D];
-  __shared__ int s_fail;
+  constexpr int CPR = D / 8;                 // 16-byte chunks per row
+  constexpr int KS = D / 16;                 // k-steps of Q K^T
+  constexpr int NT = D / 8;                  // 8-channel tiles of the output
+  constexpr int kRowBytes = D * 2;
+  extern __shared__ __align__(128) unsigned char dec_smem[];   // K rows [kDecKeys][D] swizzled, then V rows
   const int bh = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int sub = lane / LPK, ch = (lane % LPK) * 8, grp = warp * KPW + sub;
   const int n_keys = a.n_list + a.n_ring;
   const int k_lo = split * kDecKeys, k_hi = min(n_keys, k_lo + kDecKeys), nk = k_hi - k_lo;
   const int b = bh / a.Hkv, hkv = bh % a.Hkv;
-  __nv_bfloat16* sK = reinterpret_cast<__nv_bfloat16*>(dec_smem);
-  __nv_bfloat16* sV = sK + kDecKeys * D;
-  if (tid == 0) {
-    s_fail = 0;
-    ptx::mbar_init(ptx::smem_u32(&bar), 1);
-    ptx::fence_barrier_init();
-    ptx::mbar_expect_tx(ptx::smem_u32(&bar), (uint32_t)nk * D * 2 * 2);
-    const __nv_bfloat16* kl = a.k_list + (size_t)bh * a.rows_list * D;
-    const __nv_bfloat16* vl = a.v_list + (size_t)bh * a.rows_list * D;
-    const __nv_bfloat16* kr = a.k_ring + (size_t)bh * 2 * a.L * D;
-    const __nv_bfloat16* vr = a.v_ring + (size_t)bh * 2 * a.L * D;
-    int i = k_lo;
-    while (i < k_hi) {
-      const __nv_bfloat16 *ks, *vs;
-      int run;
-      if (i < a.n_list) {
-        run = min(k_hi, a.n_list) - i;
-        ks = kl + (size_t)i * D; vs = vl + (size_t)i * D;
-      } else {
-        const int r = (a.ring0 + (i - a.n_list)) % (2 * a.L);
-        run = min(k_hi - i, 2 * a.L - r);
-        ks = kr + (size_t)r * D; vs = vr + (size_t)r * D;
-      }
-      const uint32_t bytes = (uint32_t)run * D * 2;
-      bulk_load(ptx::smem_u32(sK + (size_t)(i - k_lo) * D), ks, bytes, ptx::smem_u32(&bar));
-      bulk_load(ptx::smem_u32(sV + (size_t)(i - k_lo) * D), vs, bytes, ptx::smem_u32(&bar));
-      i += run;
-    }
-  }
-  __syncthreads();
-  {
-    // bounded wait for the copies; a CTA that gives up records it and leaves its partial result empty
-    bool ok = ptx::mbar_try_wait(ptx::smem_u32(&bar), 0);
-    const long long t0 = clock64();
-    while (!ok) {
-      ok = ptx::mbar_try_wait(ptx::smem_u32(&bar), 0);
-      if (!ok && clock64() - t0 > 4000000000LL) { s_fail = 1; break; }
-    }
-  }
-  __syncthreads();
-  const bool failed = s_fail != 0;
-  if (failed && tid == 0) atomicExch(a.status, (int)LRSA_ERR_TIMEOUT);
+  const uint32_t sK = ptx::smem_u32(dec_smem), sV = sK + kDecKeys * kRowBytes;
+  // chunk c of row r sits at chunk (c & ~7) | ((c ^ r) & 7)
+  auto swz = [](int r, int c) { return (uint32_t)(r * kRowBytes + (((c & ~7) | ((c ^ r) & 7)) << 4)); };
 
+  {
+    // this thread's row of K and of V
+    const int r = tid;
+    if (r < nk) {
+      const int k = k_lo + r;
+      const __nv_bfloat16 *ks, *vs;
+      if (k < a.n_list) {
+        const size_t off = ((size_t)bh * a.rows_list + k) * D;
+        ks = a.k_list + off; vs = a.v_list + off;
+      } else {
+        const size_t off = ((size_t)bh * 2 * a.L + (a.ring0 + (k - a.n_list)) % (2 * a.L)) * D;
+        ks = a.k_ring + off; vs = a.v_ring + off;
+      }
+#pragma unroll
+      for (int c = 0; c < CPR; ++c) {
+        cp_async16(sK + swz(r, c), ks + c * 8);
+        cp_async16(sV + swz(r, c), vs + c * 8);
+      }
+    } else {
+      // rows beyond the split's keys: their probabilities are zero, their V must not be NaN
+#pragma unroll
+      for (int c = 0; c < CPR; ++c) {
+        *reinterpret_cast<uint4*>(dec_smem + swz(r, c)) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(dec_smem + kDecKeys * kRowBytes + swz(r, c)) = make_uint4(0, 0, 0, 0);
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+
+  const int row = lane >> 2, cpair = (lane & 3) * 2;   // fragment coordinates of this lane
   for (int g0 = 0; g0 < a.G; g0 += kDecHeads) {
     const int ng = min(kDecHeads, a.G - g0);
-    float q[kDecHeads][8], acc[kDecHeads][8], m[kDecHeads], l[kDecHeads];
+    // Q as A fragments: rows = heads g0 + row and g0 + row + 8, straight from global memory
+    uint32_t qa[KS][4];
+    {
+      const __nv_bfloat16* qb = a.q + ((size_t)(b * a.Hq + hkv * a.G + g0)) * D;
 #pragma unroll
-    for (int g = 0; g < kDecHeads; ++g) {
-      m[g] = -INFINITY; l[g] = 0.f;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) { acc[g][e] = 0.f; q[g][e] = 0.f; }
-      if (g < ng) {
-        const uint4 x = *reinterpret_cast<const uint4*>(a.q + ((size_t)(b * a.Hq + hkv * a.G + g0 + g)) * D + ch);
-        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) { q[g][2 * e] = bf_lo(w[e]) * a.scale_log2; q[g][2 * e + 1] = bf_hi(w[e]) * a.scale_log2; }
+      for (int ks = 0; ks < KS; ++ks) {
+        const int c0 = ks * 16 + cpair;
+        qa[ks][0] = row < ng ? *reinterpret_cast<const uint32_t*>(qb + (size_t)row * D + c0) : 0u;
+        qa[ks][1] = row + 8 < ng ? *reinterpret_cast<const uint32_t*>(qb + (size_t)(row + 8) * D + c0) : 0u;
+        qa[ks][2] = row < ng ? *reinterpret_cast<const uint32_t*>(qb + (size_t)row * D + c0 + 8) : 0u;
+        qa[ks][3] = row + 8 < ng ? *reinterpret_cast<const uint32_t*>(qb + (size_t)(row + 8) * D + c0 + 8) : 0u;
       }
     }
-    for (int i0 = warp * KPW; i0 < nk && !failed; i0 += (kDecThreads / 32) * KPW) {
-      const int i = i0 + sub;
-      const bool live = i < nk;
-      uint4 kx = make_uint4(0, 0, 0, 0), vx = make_uint4(0, 0, 0, 0);
-      if (live) {
-        kx = *reinterpret_cast<const uint4*>(sK + (size_t)i * D + ch);
-        vx = *reinterpret_cast<const uint4*>(sV + (size_t)i * D + ch);
+    if (g0 == 0) {
+      asm volatile("cp.async.wait_all;" ::: "memory");
+      __syncthreads();
+    }
+    // S = Q K^T for this warp's 32 keys: four tiles of 8 keys
+    float s[4][4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+      const int key = warp * 32 + 8 * j + (lane & 7);
+#pragma unroll
+      for (int q4 = 0; q4 < CPR / 4; ++q4) {
+        uint32_t kb[4];
+        ldmatrix_x4(sK + swz(key, 4 * q4 + (lane >> 3)), kb);
+        mma_16816(s[j], qa[2 * q4], kb[0], kb[1]);
+        mma_16816(s[j], qa[2 * q4 + 1], kb[2], kb[3]);
       }
-      const uint32_t kw[4] = {kx.x, kx.y, kx.z, kx.w}, vw[4] = {vx.x, vx.y, vx.z, vx.w};
-      float kf[8], vf[8];
+    }
+    // scale, mask the keys beyond the split, row maxima and sums (rows: head `row` -> index 0, `row + 8` -> 1)
+    float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        kf[2 * e] = bf_lo(kw[e]); kf[2 * e + 1] = bf_hi(kw[e]);
-        vf[2 * e] = bf_lo(vw[e]); vf[2 * e + 1] = bf_hi(vw[e]);
+        const int key = warp * 32 + 8 * j + cpair + (e & 1);
+        s[j][e] = key < nk ? s[j][e] * a.scale_log2 : -INFINITY;
+        mx[e >> 1] = fmaxf(mx[e >> 1], s[j][e]);
       }
 #pragma unroll
-      for (int g = 0; g < kDecHeads; ++g) {
-        if (g < ng) {   // uniform over the CTA
-          float s = 0.f;
-#pragma unroll
-          for (int e = 0; e < 8; ++e) s = fmaf(q[g][e], kf[e], s);
-#pragma unroll
-          for (int o = LPK / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-          if (live) {
-            const float mn = fmaxf(m[g], s);
-            const float f = exp2f(m[g] - mn), pr = exp2f(s - mn);   // exp2f(-inf) = 0 on the first key
-            l[g] = l[g] * f + pr;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[g][e] = fmaf(acc[g][e], f, pr * vf[e]);
-            m[g] = mn;
-          }
-        }
-      }
+    for (int h = 0; h < 2; ++h) {
+      mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+      mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
     }
-    // merge the lane groups of the CTA: one head at a time through shared memory
-    for (int g = 0; g < ng; ++g) {
-      __syncthreads();
-      if (lane % LPK == 0) { red_m[grp][g] = m[g]; red_l[grp][g] = l[g]; }
+    float sum[2] = {0.f, 0.f};
+    uint32_t pa[2][4];   // P as A fragments of the two 16-key steps
 #pragma unroll
-      for (int e = 0; e < 8; ++e) red_o[grp][ch + e] = acc[g][e];
-      __syncthreads();
-      if (tid < D) {
-        float M = -INFINITY;
-        for (int r = 0; r < kGroups; ++r) M = fmaxf(M, red_m[r][g]);
-        float o = 0.f, lsum = 0.f;
-        for (int r = 0; r < kGroups; ++r) {
-          const float f = red_m[r][g] == -INFINITY ? 0.f : exp2f(red_m[r][g] - M);
-          o = fmaf(red_o[r][tid], f, o);
-          lsum = fmaf(red_l[r][g], f, lsum);
-        }
-        float* dst = a.part + (((size_t)bh * a.n_split + split) * a.G + g0 + g) * (D + 2);
-        dst[tid] = o;
-        if (tid == 0) { dst[D] = M; dst[D + 1] = lsum; }
+    for (int j = 0; j < 4; ++j) {
+      float pr[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        pr[e] = mx[e >> 1] == -INFINITY ? 0.f : exp2f(s[j][e] - mx[e >> 1]);
+        sum[e >> 1] += pr[e];
       }
+      pa[j >> 1][(j & 1) * 2 + 0] = ptx::pack_bf16(pr[0], pr[1]);
+      pa[j >> 1][(j & 1) * 2 + 1] = ptx::pack_bf16(pr[2], pr[3]);
     }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      sum[h] += __shfl_xor_sync(0xffffffffu, sum[h], 1);
+      sum[h] += __shfl_xor_sync(0xffffffffu, sum[h], 2);
+    }
+    // O = P V: V fragments transposed on the way out of shared memory (keys are the contraction index)
+    float o[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+      uint32_t vb[4];
+      ldmatrix_x4_trans(sV + swz(warp * 32 + lane, nt), vb);
+      mma_16816(o[nt], pa[0], vb[0], vb[1]);
+      mma_16816(o[nt], pa[1], vb[2], vb[3]);
+    }
+    // merge the four warps through shared memory (the K rows are no longer needed once every warp is here;
+    // with more than one pass over the heads they are needed again, so the merge buffer then follows V)
+    __syncthreads();
+    float* mrg = reinterpret_cast<float*>(dec_smem + (a.G > kDecHeads ? 2 * kDecKeys * kRowBytes : 0));
+    float* mo = mrg;                                   // [4 warps][16 heads][D]
+    float* mm_ = mrg + 4 * kDecHeads * D;              // [4][16] maxima
+    float* ml = mm_ + 4 * kDecHeads;                   // [4][16] sums
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      *reinterpret_cast<float2*>(mo + ((warp * kDecHeads + row) * D + nt * 8 + cpair)) = make_float2(o[nt][0], o[nt][1]);
+      *reinterpret_cast<float2*>(mo + ((warp * kDecHeads + row + 8) * D + nt * 8 + cpair)) = make_float2(o[nt][2], o[nt][3]);
+    }
+    if ((lane & 3) == 0) {
+      mm_[warp * kDecHeads + row] = mx[0]; mm_[warp * kDecHeads + row + 8] = mx[1];
+      ml[warp * kDecHeads + row] = sum[0]; ml[warp * kDecHeads + row + 8] = sum[1];
+    }
+    __syncthreads();
+    for (int i = tid; i < ng * D; i += kDecThreads) {
+      const int g = i / D, c = i % D;
+      float M = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) M = fmaxf(M, mm_[w * kDecHeads + g]);
+      float ov = 0.f, lsum = 0.f;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const float mw = mm_[w * kDecHeads + g];
+        const float f = mw == -INFINITY ? 0.f : exp2f(mw - M);
+        ov = fmaf(mo[(w * kDecHeads + g) * D + c], f, ov);
+        lsum = fmaf(ml[w * kDecHeads + g], f, lsum);
+      }
+      float* dst = a.part + (((size_t)bh * a.n_split + split) * a.G + g0 + g) * (D + 2);
+      dst[c] = ov;
+      if (c == 0) { dst[D] = M; dst[D + 1] = lsum; }
+    }
+    __syncthreads();   // the merge buffer is reused by the next pass
   }
 }
 
 // One CTA per (batch, query head): merges the partial results of the splits.  kMergeRows thread rows take
-// alternate splits (so their loads are in flight together), then the rows are merged through shared memory.
+// alternate splits, four at a time with all their loads issued before the arithmetic (the kernel is a chain of
+// L2 round trips otherwise), then the rows are merged through shared memory.
 constexpr int kMergeRows = 8;
 template <int D>
 __global__ void __launch_bounds__(kMergeRows * D) decode_merge_kernel(const float* __restrict__ part,
@@ -258,12 +303,29 @@ __global__ void __launch_bounds__(kMergeRows * D) decode_merge_kernel(const floa
   const float* base = part + (((size_t)(b * Hkv + hkv) * n_split) * G + g) * (D + 2);
   const size_t stride = (size_t)G * (D + 2);
   float M = -INFINITY, acc = 0.f, l = 0.f;
-  for (int s = row; s < n_split; s += kMergeRows) {
-    const float ms = base[s * stride + D];
-    if (ms == -INFINITY) continue;
-    const float mn = fmaxf(M, ms), f0 = exp2f(M - mn), f1 = exp2f(ms - mn);
-    acc = acc * f0 + base[s * stride + c] * f1;
-    l = l * f0 + base[s * stride + D + 1] * f1;
+  constexpr int kBatch = 4;
+  for (int s0 = row; s0 < n_split; s0 += kMergeRows * kBatch) {
+    float ms[kBatch], vs[kBatch], ls[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int s = s0 + u * kMergeRows;
+      const bool in = s < n_split;
+      ms[u] = in ? __ldcg(base + s * stride + D) : -INFINITY;
+      vs[u] = in ? __ldcg(base + s * stride + c) : 0.f;
+      ls[u] = in ? __ldcg(base + s * stride + D + 1) : 0.f;
+    }
+    float mn = M;
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) mn = fmaxf(mn, ms[u]);
+    if (mn == -INFINITY) continue;
+    const float f0 = exp2f(M - mn);   // exp2f(-inf) = 0 while nothing has been merged
+    acc *= f0; l *= f0;
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const float f = exp2f(ms[u] - mn);
+      acc = fmaf(vs[u], f, acc);
+      l = fmaf(ls[u], f, l);
+    }
     M = mn;
   }
   sm_o[row][c] = acc;
@@ -432,7 +494,11 @@ int lrsa_attn_decode(const lrsa_params_t* params, const void* cache, size_t cach
   LRSA_CUDA_CHECK(cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st));
   launch_counter().n++;
   const dim3 grid(a.n_split, a.BHkv);
-  const size_t smem = (size_t)2 * kDecKeys * g.d * sizeof(__nv_bfloat16);
+  // K and V rows; the merge buffer (4 warps x 16 heads x (d + 2) floats) lies over them, or behind them when the
+  // group has more than 16 query heads and the rows are read again
+  const size_t rows_bytes = (size_t)2 * kDecKeys * g.d * sizeof(__nv_bfloat16);
+  const size_t merge_bytes = (size_t)4 * kDecHeads * (g.d + 2) * sizeof(float);
+  const size_t smem = g.G > kDecHeads ? rows_bytes + merge_bytes : (rows_bytes > merge_bytes ? rows_bytes : merge_bytes);
   if (g.d == 128) {
     LRSA_CUDA_CHECK(cudaFuncSetAttribute(decode_partial_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     decode_partial_kernel<128><<<grid, kDecThreads, smem, st>>>(a);
