@@ -141,6 +141,11 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const Decod
   const int k_lo = split * kDecKeys, k_hi = min(n_keys, k_lo + kDecKeys), nk = k_hi - k_lo;
   const int b = bh / a.Hkv, hkv = bh % a.Hkv;
   const uint32_t sK = ptx::smem_u32(dec_smem), sV = sK + kDecKeys * kRowBytes;
+  // The merge kernel is launched as a programmatic dependent of this one: its CTAs may be scheduled from here
+  // on and wait (griddepcontrol.wait) until this grid has completed and its stores are visible.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // Nothing in this call writes the status word but this store (no wait here can expire).
+  if (tid == 0 && split == 0 && bh == 0) *a.status = 0;
   // chunk c of row r sits at chunk (c & ~7) | ((c ^ r) & 7)
   auto swz = [](int r, int c) { return (uint32_t)(r * kRowBytes + (((c & ~7) | ((c ^ r) & 7)) << 4)); };
 
@@ -304,6 +309,8 @@ __global__ void __launch_bounds__(kMergeRows * D) decode_merge_kernel(const floa
   const size_t stride = (size_t)G * (D + 2);
   float M = -INFINITY, acc = 0.f, l = 0.f;
   constexpr int kBatch = 4;
+  // launched as a programmatic dependent of the partial kernel: wait for its grid to complete
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   for (int s0 = row; s0 < n_split; s0 += kMergeRows * kBatch) {
     float ms[kBatch], vs[kBatch], ls[kBatch];
 #pragma unroll
@@ -491,8 +498,6 @@ int lrsa_attn_decode(const lrsa_params_t* params, const void* cache, size_t cach
   a.n_split = decode_splits(a.n_list + a.n_ring);
   a.scale_log2 = g.scale * 1.4426950408889634f;
   a.status = &reinterpret_cast<WsHeader*>(workspace)->status;
-  LRSA_CUDA_CHECK(cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st));
-  launch_counter().n++;
   const dim3 grid(a.n_split, a.BHkv);
   // K and V rows; the merge buffer (4 warps x 16 heads x (d + 2) floats) lies over them, or behind them when the
   // group has more than 16 query heads and the rows are read again
@@ -508,10 +513,25 @@ int lrsa_attn_decode(const lrsa_params_t* params, const void* cache, size_t cach
   }
   LRSA_CUDA_CHECK(cudaGetLastError());
   launch_counter().n++;
-  if (g.d == 128)
-    decode_merge_kernel<128><<<g.B * g.Hq, kMergeRows * 128, 0, st>>>(a.part, static_cast<__nv_bfloat16*>(o), lse, g.Hq, g.Hkv, g.G, a.n_split);
-  else
-    decode_merge_kernel<64><<<g.B * g.Hq, kMergeRows * 64, 0, st>>>(a.part, static_cast<__nv_bfloat16*>(o), lse, g.Hq, g.Hkv, g.G, a.n_split);
+  {
+    // programmatic dependent launch: the merge kernel's launch latency overlaps the partial kernel
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(g.B * g.Hq);
+    cfg.blockDim = dim3(kMergeRows * g.d);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const float* part = a.part;
+    __nv_bfloat16* op = static_cast<__nv_bfloat16*>(o);
+    if (g.d == 128)
+      LRSA_CUDA_CHECK(cudaLaunchKernelEx(&cfg, decode_merge_kernel<128>, part, op, lse, g.Hq, g.Hkv, g.G, a.n_split));
+    else
+      LRSA_CUDA_CHECK(cudaLaunchKernelEx(&cfg, decode_merge_kernel<64>, part, op, lse, g.Hq, g.Hkv, g.G, a.n_split));
+  }
   LRSA_CUDA_CHECK(cudaGetLastError());
   launch_counter().n++;
   return LRSA_OK;
