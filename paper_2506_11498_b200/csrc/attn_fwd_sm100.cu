@@ -1,19 +1,22 @@
 // LRSA attention forward on tcgen05 tensor cores (Section 3.1 Eq. 3 under the chunked mask of
 // Section 3.2).
 //
-// A CTA owns one 128-row query tile of one (batch, query head) and walks its key list (first n_front
-// rows of the compact sinks+kept buffer, then a contiguous range of original positions up to the
-// diagonal) in 128-key tiles.  Q is copied once into tensor memory, so both products take their
-// 128-row operand from TMEM and only K_j / V_j from shared memory.  Roles:
-//   warp 0      TMA producer: the Q tile once, then K_j, V_j tiles through a ring of shared-memory slots
-//   warp 1      issues S_j = Q K_j^T into one of two TMEM buffers; owns the TMEM allocation
-//   warp 2      issues O += P_j V_j with P_j read from tensor memory
-//   warps 4-11  softmax: both warpgroups work on every tile, 64 key columns each; S from TMEM, online
-//               softmax in fp32 with the maximum only raised when it grew by more than 2^8 (then O is
+// A CTA owns up to 256 query rows of one (batch, query head) that share a key list (two 128-row tiles of
+// one query chunk) and walks the list (first n_front rows of the compact sinks+kept buffer, then a contiguous
+// range of original positions up to the diagonal) in 128-key tiles; every K_j / V_j tile in shared memory
+// serves both query tiles.  Roles:
+//   warp 0      TMA producer: the Q tiles once, then K_j, V_j tiles through a ring of shared-memory slots
+//   warp 1      issues S_t = Q_t K_j^T (both operands in shared memory) into the tile's TMEM region; owns
+//               the TMEM allocation
+//   warp 2      issues O_t += P_t V_j with P_t read from tensor memory
+//   warps 4-7   softmax of query tile 0, warps 8-11 of query tile 1: one thread per row, S from TMEM, online
+//               softmax in fp32 with the maximum only raised when it grew by more than 2^8 (then O_t is
 //               rescaled in TMEM), P written back over S as packed bf16
-// S is double-buffered, so the tensor core computes S_{j+1} while tile j is in the softmax.  The
-// issuing warps run their loops with all lanes and elect one lane per instruction.  All mbarrier
-// waits are bounded; on expiry the CTA records LRSA_ERR_TIMEOUT in the workspace header and leaves.
+// The two tiles take turns on the tensor core: while one tile's scores are in its softmax warpgroup the
+// products of the other run.  A row belongs to one thread from its scores to its output, so the softmax
+// threads exchange nothing.  The issuing warps run their loops with all lanes and elect one lane per
+// instruction.  All mbarrier waits are bounded; on expiry the CTA records LRSA_ERR_TIMEOUT in the workspace
+// header and leaves.
 #include "attn_common_sm100.h"
 
 namespace lrsa {
@@ -26,15 +29,18 @@ struct FwdCfg {
   static constexpr int kSub = D / 64;                 // 64-column (128-byte) sub-tiles per tile
   static constexpr int kSubBytes = kTile * 128;       // 16 KB
   static constexpr int kTileBytes = kSub * kSubBytes; // one Q / K / V tile
-  static constexpr int kStages = D == 128 ? 6 : 12;   // K/V ring slots
-  static constexpr int kSmem = (1 + kStages) * kTileBytes + 1024;
+  // A Q tile is followed by 2 KB so that the output rows of the tile can be staged there with 16 bytes of
+  // padding per row (128 rows x (2D + 16) bytes = tile + 2 KB); the next tile stays 1024-byte aligned.
+  static constexpr int kQRegion = kTileBytes + 2048;
+  static constexpr int kStages = D == 128 ? 4 : 10;   // K/V ring slots
+  static constexpr int kSmem = 2 * kQRegion + kStages * kTileBytes + 1024;
   static constexpr int kThreads = 384;
-  // TMEM columns: Q as packed bf16 (D/2 columns), the accumulator O at 64, S buffer b at 256 + 128b
-  static constexpr uint32_t kColQ = 0, kColO = 64, kColS = 256;
+  // TMEM columns: accumulator O of query tile t at 128t, its S (and, packed over it, P) at 256 + 128t
+  static constexpr uint32_t kColO = 0, kColS = 256;
 };
 
 struct FwdArgs {
-  BlockPlan plan;
+  BlockPlan plan;          // blocks of up to 256 query rows (two tiles)
   int BH, Hq, Hkv, G, N;   // N: tokens per (batch, head) row of O and LSE (the row stride)
   __nv_bfloat16* O;
   __nv_bfloat16* Olo;        // optional: receives bf16(O_fp32 - O), the part of the output the bf16 O cannot hold
@@ -44,9 +50,9 @@ struct FwdArgs {
 };
 
 struct FwdBars {
-  uint64_t q_full, qt_ready, pv_done;
+  uint64_t q_full;
   uint64_t kv_full[12], kv_empty[12];
-  uint64_t s_full[2], p_full[2], buf_free[2];
+  uint64_t s_full[2], p_full[2], buf_free[2], pv_done[2];   // per query tile
 };
 
 template <int D>
@@ -58,35 +64,34 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   constexpr int NS = Cfg::kStages;
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) FwdBars bars;
-  __shared__ float red_s[2][kTile];   // [column half][row] partial row sums
-  __shared__ unsigned short loaded_s[2][kTile];   // [column half][row] tiles whose S this softmax thread has read
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sQ = smem0, sRing = smem0 + Cfg::kTileBytes;
+  const uint32_t sQ = smem0, sRing = smem0 + 2 * Cfg::kQRegion;
 
   const int bh = blockIdx.x % a.BH, blk = blockIdx.x / a.BH;
   const RowBlock rb = decode_block(a.plan, blk);
   const int bh_kv = (bh / a.Hq) * a.Hkv + (bh % a.Hq) / a.G;
   const int n_ct = (rb.n_front + kTile - 1) / kTile;
-  const int n = n_ct + (rb.q_end - 1 - rb.dense_start) / kTile + 1;   // key tiles of this block (>= 1)
+  // key tiles of query tile t: the list, then the dense range up to the tile's last row (0: the tile is empty)
+  const int n0 = n_ct + (min(rb.q_end, rb.q0 + kTile) - 1 - rb.dense_start) / kTile + 1;
+  const int n1 = rb.q0 + kTile < rb.q_end ? n_ct + (rb.q_end - 1 - rb.dense_start) / kTile + 1 : 0;
+  const int n = max(n0, n1);
 
   if (tid == 0) {
     abort_s = 0;
     mbar_init(smem_u32(&bars.q_full), 1);
-    mbar_init(smem_u32(&bars.qt_ready), 256);
-    mbar_init(smem_u32(&bars.pv_done), 1);
     for (int i = 0; i < NS; ++i) { mbar_init(smem_u32(&bars.kv_full[i]), 1); mbar_init(smem_u32(&bars.kv_empty[i]), 1); }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&bars.s_full[b]), 1);
-      mbar_init(smem_u32(&bars.p_full[b]), 256);    // every softmax thread
-      mbar_init(smem_u32(&bars.buf_free[b]), 1);
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(smem_u32(&bars.s_full[t]), 1);
+      mbar_init(smem_u32(&bars.p_full[t]), 128);    // every softmax thread of the tile's warpgroup
+      mbar_init(smem_u32(&bars.buf_free[t]), 1);
+      mbar_init(smem_u32(&bars.pv_done[t]), 1);
     }
     fence_barrier_init();
   }
-  if (tid < 2 * kTile) (&loaded_s[0][0])[tid] = 0;
   if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_s), 512); tmem_relinquish(); }
   tc_fence_before_sync();
   __syncthreads();
@@ -99,9 +104,10 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     if (lane == 0) {
       prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV);
       prefetch_tensormap(&mapKc); prefetch_tensormap(&mapVc);
-      mbar_expect_tx(smem_u32(&bars.q_full), Cfg::kTileBytes);
-      for (int h = 0; h < Cfg::kSub; ++h)
-        tma_load_3d(sQ + h * Cfg::kSubBytes, &mapQ, h * 64, rb.q0, bh, smem_u32(&bars.q_full));
+      mbar_expect_tx(smem_u32(&bars.q_full), (n1 > 0 ? 2 : 1) * Cfg::kTileBytes);
+      for (int t = 0; t < (n1 > 0 ? 2 : 1); ++t)
+        for (int h = 0; h < Cfg::kSub; ++h)
+          tma_load_3d(sQ + t * Cfg::kQRegion + h * Cfg::kSubBytes, &mapQ, h * 64, rb.q0 + t * kTile, bh, smem_u32(&bars.q_full));
       int it = 0;
       bool ok = true;
       for (int j = 0; j < n && ok; ++j) {
@@ -128,131 +134,122 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       }
     }
   } else if (warp == 1) {
-    // ---------------- S issuer: S_j = Q K_j^T into buffer j & 1 ----------------
+    // ---------------- S issuer: S_t = Q_t K_j^T for both query tiles ----------------
     constexpr uint32_t idesc_qk = make_idesc_bf16(kTile, kTile, 0, 0);
     const uint64_t descK0 = make_smem_desc_sw128(sRing, 16, 1024);
-    bool ok = mbar_wait_warp(smem_u32(&bars.qt_ready), 0, abort);   // Q is in tensor memory
+    const uint64_t descQ0 = make_smem_desc_sw128(sQ, 16, 1024);
+    bool ok = mbar_wait_warp(smem_u32(&bars.q_full), 0, abort);
     for (int j = 0; j < n && ok; ++j) {
-      const int it = 2 * j, b = j & 1;   // ring order: K_j at 2j, V_j at 2j+1
+      const int it = 2 * j;   // ring order: K_j at 2j, V_j at 2j+1
       ok = mbar_wait_warp(smem_u32(&bars.kv_full[it % NS]), (it / NS) & 1, abort);
-      if (ok && j >= 2) ok = mbar_wait_warp(smem_u32(&bars.buf_free[b]), ((j >> 1) - 1) & 1, abort);
-      if (!ok) break;
-      tc_fence_after_sync();
       const uint64_t dK = desc_advance(descK0, (it % NS) * Cfg::kTileBytes);
+      for (int t = 0; t < 2 && ok; ++t) {
+        if (j >= (t == 0 ? n0 : n1)) continue;
+        // S_t is also where P_t lives: the tile's previous O += P V must have read it
+        if (j >= 1) ok = mbar_wait_warp(smem_u32(&bars.buf_free[t]), (j - 1) & 1, abort);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint64_t dQ = desc_advance(descQ0, t * Cfg::kQRegion);
 #pragma unroll
-      for (int kk = 0; kk < D / 16; ++kk) {
-        const uint64_t bd = desc_advance(dK, (kk >> 2) * Cfg::kSubBytes + (kk & 3) * 32);
-        if (elect_one()) umma_ts(tmem + Cfg::kColS + b * kTile, tmem + Cfg::kColQ + kk * 8, bd, idesc_qk, kk > 0 ? 1u : 0u);
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * Cfg::kSubBytes + (kk & 3) * 32;
+          const uint64_t ad = desc_advance(dQ, off), bd = desc_advance(dK, off);
+          if (elect_one()) umma_ss(tmem + Cfg::kColS + t * kTile, ad, bd, idesc_qk, kk > 0 ? 1u : 0u);
+        }
+        if (elect_one()) umma_commit(smem_u32(&bars.s_full[t]));
+        __syncwarp();
       }
-      if (elect_one()) {
-        umma_commit(smem_u32(&bars.s_full[b]));
-        umma_commit(smem_u32(&bars.kv_empty[it % NS]));   // K_j is used by S_j only
-      }
+      if (ok && elect_one()) umma_commit(smem_u32(&bars.kv_empty[it % NS]));   // K_j is used by the S products only
       __syncwarp();
     }
   } else if (warp == 2) {
-    // ---------------- O issuer: O += P_j V_j ----------------
+    // ---------------- O issuer: O_t += P_t V_j ----------------
     constexpr uint32_t idesc_pv = make_idesc_bf16(kTile, D, 0, 1);
     const uint64_t descV0 = make_smem_desc_sw128(sRing, Cfg::kSubBytes, 1024);   // V_j MN-major
     bool ok = true;
     for (int j = 0; j < n && ok; ++j) {
-      const int it = 2 * j + 1, b = j & 1;
+      const int it = 2 * j + 1;
       ok = mbar_wait_warp(smem_u32(&bars.kv_full[it % NS]), (it / NS) & 1, abort);
-      if (ok) ok = mbar_wait_warp(smem_u32(&bars.p_full[b]), (j >> 1) & 1, abort);
-      if (!ok) break;
-      tc_fence_after_sync();
       const uint64_t dV = desc_advance(descV0, (it % NS) * Cfg::kTileBytes);
-      const uint32_t acc0 = j > 0 ? 1u : 0u;
-      // packed P: keys [0,64) in columns [0,32) of the buffer, keys [64,128) in columns [64,96)
+      for (int t = 0; t < 2 && ok; ++t) {
+        if (j >= (t == 0 ? n0 : n1)) continue;
+        ok = mbar_wait_warp(smem_u32(&bars.p_full[t]), j & 1, abort);
+        if (!ok) break;
+        tc_fence_after_sync();
+        // packed P_t: keys [16k, 16k+16) in columns [8k, 8k+8) of the tile's S region
 #pragma unroll
-      for (int kk = 0; kk < kTile / 16; ++kk) {
-        const uint64_t bd = desc_advance(dV, kk * 2048);
-        if (elect_one())
-          umma_ts(tmem + Cfg::kColO, tmem + Cfg::kColS + b * kTile + (kk >> 2) * 64 + (kk & 3) * 8, bd, idesc_pv,
-                  kk > 0 ? 1u : acc0);
+        for (int kk = 0; kk < kTile / 16; ++kk) {
+          const uint64_t bd = desc_advance(dV, kk * 2048);
+          if (elect_one())
+            umma_ts(tmem + Cfg::kColO + t * kTile, tmem + Cfg::kColS + t * kTile + kk * 8, bd, idesc_pv,
+                    (kk > 0 || j > 0) ? 1u : 0u);
+        }
+        if (elect_one()) {
+          umma_commit(smem_u32(&bars.buf_free[t]));    // S_t of the next key tile may overwrite P_t
+          umma_commit(smem_u32(&bars.pv_done[t]));     // phase j: O_t holds key tiles 0..j
+        }
+        __syncwarp();
       }
-      if (elect_one()) {
-        umma_commit(smem_u32(&bars.kv_empty[it % NS]));
-        umma_commit(smem_u32(&bars.buf_free[b]));     // tile j+2 may overwrite the buffer
-        umma_commit(smem_u32(&bars.pv_done));         // phase j: O holds tiles 0..j
-      }
+      if (ok && elect_one()) umma_commit(smem_u32(&bars.kv_empty[it % NS]));
       __syncwarp();
     }
   } else if (warp >= 4) {
-    // ---------------- softmax + epilogue: warpgroup `half` takes key columns [64*half, 64*half+64) ----------------
-    const int half = (warp - 4) >> 2, quad = warp & 3;
+    // ---------------- softmax + epilogue: warpgroup t owns query tile t, one thread per row ----------------
+    const int t = (warp - 4) >> 2, quad = warp & 3;
     const int row = quad * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const uint32_t O_addr = tmem + lane_addr + Cfg::kColO + half * (D / 2);   // this thread's half of the O columns
-    const int qpos = rb.q0 + row;
+    const uint32_t S_addr = tmem + lane_addr + Cfg::kColS + t * kTile;
+    const uint32_t O_addr = tmem + lane_addr + Cfg::kColO + t * kTile;
+    const int nt = t == 0 ? n0 : n1;
+    const int qpos = rb.q0 + t * kTile + row;
     const float c = a.scale_log2;
-    // copy this thread's row of one 64-column sub-tile of Q from the swizzled shared-memory tile into
-    // tensor memory: 16-byte chunk ch of row r sits at chunk ch ^ (r & 7)
-    bool ok = mbar_wait(smem_u32(&bars.q_full), 0, abort);
-    if (ok && half < Cfg::kSub) {
-      const unsigned char* src = smem_raw + (sQ - smem_u32(smem_raw)) + half * Cfg::kSubBytes + row * 128;
-      uint32_t v[32];
-#pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        const uint4 x = *reinterpret_cast<const uint4*>(src + ((ch ^ (row & 7)) << 4));
-        v[4 * ch] = x.x; v[4 * ch + 1] = x.y; v[4 * ch + 2] = x.z; v[4 * ch + 3] = x.w;
-      }
-      tmem_st32(tmem + lane_addr + Cfg::kColQ + half * 32, v);
-      tmem_wait_st();
-    }
-    tc_fence_before_sync();
-    mbar_arrive(smem_u32(&bars.qt_ready));   // also when the wait gave up: the issuers then see abort
-    float m = -INFINITY, l = 0.f;
-    volatile unsigned short* my_loaded = &loaded_s[half][row];
-    volatile unsigned short* partner_loaded = &loaded_s[1 - half][row];
-    for (int j = 0; j < n && ok; ++j) {
-      const int b = j & 1;
-      ok = mbar_wait(smem_u32(&bars.s_full[b]), (j >> 1) & 1, abort);
+    float m = 0.f, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < nt && ok; ++j) {
+      ok = mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t S_own = tmem + lane_addr + Cfg::kColS + b * kTile + half * 64;
-      const uint32_t S_oth = tmem + lane_addr + Cfg::kColS + b * kTile + (1 - half) * 64;
-      uint32_t s[64], t[64];
-      tmem_ld32(S_own, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-      tmem_ld32(S_own + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
-      tmem_ld32(S_oth, *reinterpret_cast<uint32_t(*)[32]>(&t[0]));
-      tmem_ld32(S_oth + 32, *reinterpret_cast<uint32_t(*)[32]>(&t[32]));
-      tmem_wait_ld();
-      *my_loaded = (unsigned short)(j + 1);   // the partner may now overwrite its S columns of this tile with P
       // keys of the tile this row may see: the first `limit`
       const int limit = j < n_ct ? rb.n_front - j * kTile : qpos - (rb.dense_start + (j - n_ct) * kTile) + 1;
-      if (limit < kTile) {
-        const int lim_own = limit - half * 64, lim_oth = limit - (1 - half) * 64;
+      // Row maximum over the 128 columns, 64 at a time; the second half stays in registers for its
+      // exponentials, the first half is read again afterwards (a second read of tensor memory is cheaper than
+      // 64 more live registers).
+      uint32_t s[64];
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < 64; ++i) {
-          if (i >= lim_own) s[i] = 0xff800000u;  // -inf
-          if (i >= lim_oth) t[i] = 0xff800000u;
+      for (int h = 0; h < 2; ++h) {
+        tmem_ld32(S_addr + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+        tmem_ld32(S_addr + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+        tmem_wait_ld();
+        if (limit < kTile) {
+          const int lim = limit - h * 64;
+#pragma unroll
+          for (int i = 0; i < 64; ++i)
+            if (i >= lim) s[i] = 0xff800000u;  // -inf
         }
-      }
-      // row maximum over all 128 columns: both threads of a row compute the same value
-      float mx0 = fmaxf(__uint_as_float(s[0]), __uint_as_float(t[0])), mx1 = fmaxf(__uint_as_float(s[1]), __uint_as_float(t[1]));
-      float mx2 = fmaxf(__uint_as_float(s[2]), __uint_as_float(t[2])), mx3 = fmaxf(__uint_as_float(s[3]), __uint_as_float(t[3]));
 #pragma unroll
-      for (int i = 4; i < 64; i += 4) {
-        mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(t[i]));
-        mx1 = max3(mx1, __uint_as_float(s[i + 1]), __uint_as_float(t[i + 1]));
-        mx2 = max3(mx2, __uint_as_float(s[i + 2]), __uint_as_float(t[i + 2]));
-        mx3 = max3(mx3, __uint_as_float(s[i + 3]), __uint_as_float(t[i + 3]));
+        for (int i = 0; i < 64; i += 4) {
+          mx0 = fmaxf(mx0, __uint_as_float(s[i]));
+          mx1 = fmaxf(mx1, __uint_as_float(s[i + 1]));
+          mx2 = fmaxf(mx2, __uint_as_float(s[i + 2]));
+          mx3 = fmaxf(mx3, __uint_as_float(s[i + 3]));
+        }
       }
       const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
       if (j == 0) {
         m = mx == -INFINITY ? 0.f : mx;
       } else {
+        // the maximum is only raised when it grew by more than 2^8 (then O is rescaled in tensor memory)
         const bool need = (mx - m) * c > 8.f;
         if (__any_sync(0xffffffffu, need)) {
           // O must hold every earlier tile before it is rescaled; the O issuer cannot start tile j before
           // this thread has arrived on p_full, so the rescale cannot race with it
-          ok = mbar_wait(smem_u32(&bars.pv_done), (j - 1) & 1, abort);
+          ok = mbar_wait(smem_u32(&bars.pv_done[t]), (j - 1) & 1, abort);
           if (!ok) break;
           tc_fence_after_sync();
           const float f = need ? ex2((m - mx) * c) : 1.f;
 #pragma unroll
-          for (int q = 0; q < D / 64; ++q) {
+          for (int q = 0; q < D / 32; ++q) {
             uint32_t o[32];
             tmem_ld32(O_addr + q * 32, o);
             tmem_wait_ld();
@@ -268,56 +265,56 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       const float nmc = -m * c;
       const uint64_t c2 = f2_pack(c, c), nmc2 = f2_pack(nmc, nmc);
       uint64_t sum2 = f2_pack(0.f, 0.f);
-      float sum0, sum1;
-      uint32_t pk[32];
+      // exponentials of 64 columns held in s[]: scale and shift as packed pairs (one issue slot for two
+      // elements); one exponential in eight on the FMA pipe, the rest on the MUFU pipe
+      auto exps = [&](uint32_t (&pk)[32]) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        // scale and shift as packed pairs (one issue slot for two elements); one exponential in eight on
-        // the FMA pipe, the rest on the MUFU pipe (measured optimum: the polynomial costs issue slots)
-        float x0, x1;
-        f2_unpack(f2_fma(f2_pack(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), c2, nmc2), x0, x1);
-        const float p0 = ex2(x0);
-        const float p1 = (i & 3) == 3 ? ex2_fma(x1) : ex2(x1);
-        sum2 = f2_add(sum2, f2_pack(p0, p1));
-        pk[i] = pack_bf16(p0, p1);
+        for (int i = 0; i < 32; ++i) {
+          float x0, x1;
+          f2_unpack(f2_fma(f2_pack(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), c2, nmc2), x0, x1);
+          const float p0 = ex2(x0);
+          const float p1 = (i & 3) == 3 ? ex2_fma(x1) : ex2(x1);
+          sum2 = f2_add(sum2, f2_pack(p0, p1));
+          pk[i] = pack_bf16(p0, p1);
+        }
+      };
+      uint32_t pk_hi[32], pk_lo[32];
+      exps(pk_hi);   // s[] holds columns 64..127 (masked)
+      tmem_ld32(S_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+      tmem_ld32(S_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+      tmem_wait_ld();
+      if (limit < 64) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i)
+          if (i >= limit) s[i] = 0xff800000u;
       }
+      exps(pk_lo);
+      float sum0, sum1;
       f2_unpack(sum2, sum0, sum1);
       l += sum0 + sum1;
-      // The two threads of a row read each other's S columns above and overwrite their own with P below:
-      // a thread stores only after its partner has published that it has loaded this tile.  By now the
-      // partner has had a whole tile of arithmetic to do so, so the check practically never waits.
-      if ((int)*partner_loaded <= j) {
-        const long long t0 = clock64();
-        while ((int)*partner_loaded <= j) {
-          if (*abort) { ok = false; break; }
-          if (clock64() - t0 > kWaitCycles) { *abort = 1; ok = false; break; }
-        }
-      }
-      ok = __all_sync(0xffffffffu, ok);   // one verdict per warp: the store below is warp-wide
-      if (!ok) break;
-      tmem_st32(S_own, pk);   // over the first half of this warpgroup's own S columns
+      // P as packed bf16 over the first 64 columns of the tile's S (this thread's own lane: nobody else reads it)
+      tmem_st32(S_addr, pk_lo);
+      tmem_st32(S_addr + 32, pk_hi);
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(smem_u32(&bars.p_full[b]));
+      mbar_arrive(smem_u32(&bars.p_full[t]));
     }
-    red_s[half][row] = l;
-    asm volatile("bar.sync 1, 256;" ::: "memory");   // the eight softmax warps, whether or not a wait gave up
-    if (ok) ok = mbar_wait(smem_u32(&bars.pv_done), (n - 1) & 1, abort);
-    // The output rows go through shared memory (the Q tile and the first ring slot are idle by now) and
-    // leave as one bulk copy per row: per-thread 16-byte stores to rows 256 bytes apart cost a
-    // transaction each.  Rows are padded by 16 bytes so that a warp's stores spread over the banks.
+    if (ok && nt > 0) ok = mbar_wait(smem_u32(&bars.pv_done[t]), (nt - 1) & 1, abort);
+    // The output rows go through shared memory (the tile's Q region, idle once its last S product is done,
+    // which pv_done implies) and leave as one bulk copy per row: per-thread 16-byte stores to rows 256 bytes
+    // apart cost a transaction each.  Rows are padded by 16 bytes so that a warp's stores spread over the banks.
     constexpr int kRowBytes = D * 2, kStageStride = kRowBytes + 16;
-    unsigned char* stage_out = smem_raw + (sQ - smem_u32(smem_raw));
-    const bool store = qpos < rb.q_end;
-    if (ok) {
+    static_assert(kTile * kStageStride <= Cfg::kQRegion, "staging fits the Q region");
+    unsigned char* stage_out = smem_raw + (sQ - smem_u32(smem_raw)) + t * Cfg::kQRegion;
+    const bool store = qpos < rb.q_end && nt > 0;
+    if (ok && nt > 0) {
       tc_fence_after_sync();
-      const float lt = red_s[0][row] + red_s[1][row];
-      const float inv = 1.0f / lt;
-      unsigned char* srow = stage_out + row * kStageStride + half * (kRowBytes / 2);
-      // the remainder goes straight to global memory (64 or 128 contiguous bytes per thread, written once)
-      __nv_bfloat16* lo_row = a.Olo && store ? a.Olo + ((size_t)bh * a.N + qpos) * D + half * (D / 2) : nullptr;
+      const float inv = 1.0f / l;
+      unsigned char* srow = stage_out + row * kStageStride;
+      // the remainder goes straight to global memory (contiguous bytes per thread, written once)
+      __nv_bfloat16* lo_row = a.Olo && store ? a.Olo + ((size_t)bh * a.N + qpos) * D : nullptr;
 #pragma unroll
-      for (int q = 0; q < D / 64; ++q) {
+      for (int q = 0; q < D / 32; ++q) {
         uint32_t o[32];
         tmem_ld32(O_addr + q * 32, o);
         tmem_wait_ld();
@@ -340,17 +337,16 @@ lrsa_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
           }
         }
       }
-      if (store && half == 0) a.LSE[(size_t)bh * a.N + qpos] = m * a.scale + logf(lt);
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the bulk copy reads these stores
-    }
-    asm volatile("bar.sync 1, 256;" ::: "memory");   // both halves of every row are staged (or a wait gave up)
-    if (half == 0 && store && !*abort) {
-      __nv_bfloat16* orow = a.O + ((size_t)bh * a.N + qpos) * D;
-      asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(orow),
-                   "r"(smem_u32(stage_out + row * kStageStride)), "r"((uint32_t)kRowBytes)
-                   : "memory");
-      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-      asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory is released at exit
+      if (store) a.LSE[(size_t)bh * a.N + qpos] = m * a.scale + logf(l);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the bulk copy reads this thread's stores
+      if (store && !*abort) {
+        __nv_bfloat16* orow = a.O + ((size_t)bh * a.N + qpos) * D;
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(orow),
+                     "r"(smem_u32(srow)), "r"((uint32_t)kRowBytes)
+                     : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory is released at exit
+      }
     }
   }
 
@@ -468,13 +464,12 @@ static int launch_fwd_t(const Geom& g, const __nv_bfloat16* Q, const __nv_bfloat
   if (rc_ == LRSA_OK) rc_ = make_tmap_bf16(&mVc, Vc, D, rc, (long long)g.B * g.Hkv, kTile);
   if (rc_ != LRSA_OK) return rc_;
   FwdArgs a;
-  a.plan = make_plan(g, kTile);
+  a.plan = make_plan(g, 2 * kTile);
   a.BH = g.B * g.Hq; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.N = g.Nrow;
   a.O = O + sh; a.Olo = Olo ? Olo + sh : nullptr; a.LSE = LSE + g.tok0; a.scale = g.scale; a.scale_log2 = g.scale * 1.4426950408889634f;
   a.status = status;
   const long long grid = (long long)a.plan.total * a.BH;
   if (grid > 0x7fffffffLL) return LRSA_ERR_UNSUPPORTED;
-  if (g.N / kTile + 4 > 0xffff) return LRSA_ERR_UNSUPPORTED;   // 16-bit tile counters of the softmax threads
   auto kern = lrsa_fwd_kernel<D>;
   LRSA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem));
   kern<<<(unsigned)grid, Cfg::kThreads, Cfg::kSmem, st>>>(mQ, mK, mV, mKc, mVc, a);
