@@ -101,8 +101,9 @@ struct DecodeArgs {
   float scale_log2;
 };
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -120,35 +121,42 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4],
 }
 
 // Grid (n_split, BHkv).  One query token per (batch, head) and a few hundred to a few thousand keys per KV head:
-// the work is the transfer of K and V, so the CTA's (at most) 128 key rows are fetched by all threads at once
-// (one row of K and of V per thread, 16-byte asynchronous copies) and everything after that has to be short.
+// the work is the transfer of K and V, so the CTA's (at most) 128 key rows are fetched at once (every thread
+// issues one bulk copy for its row of K and one for its row of V) and everything after that has to be short.
 // The query heads of the KV group form the rows of a small matrix product (GQA: 16 rows per pass, the unused
 // ones zero), so S = Q K^T and O = P V run on the warp-level tensor-core instructions (m16n8k16, bf16 operands,
-// fp32 accumulation; a 128-row tcgen05 product would be nine tenths padding here): a warp takes 32 keys, holds
-// Q as A fragments, reads K and V fragments with ldmatrix from rows whose 16-byte chunks are XOR-swizzled by the
-// row number (rows are 128 or 256 bytes apart, eight rows of one chunk would share their banks), forms the
-// softmax of its 32 keys in registers and hands P over as the A operand of the second product.  The four
-// warps' partial results are merged through shared memory; the splits by decode_merge_kernel.
+// fp32 accumulation; a 128-row tcgen05 product would be nine tenths padding here): a warp takes 32 keys, reads
+// Q, K and V fragments with ldmatrix from rows padded by 16 bytes (rows 128 or 256 bytes apart would put the
+// eight rows of a fragment on the same banks), forms the softmax of its 32 keys in registers and hands P over
+// as the A operand of the second product.  The four warps' partial results are merged through shared memory;
+// the splits by decode_merge_kernel.
 template <int D>
 __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const DecodeArgs a) {
   constexpr int CPR = D / 8;                 // 16-byte chunks per row
   constexpr int KS = D / 16;                 // k-steps of Q K^T
   constexpr int NT = D / 8;                  // 8-channel tiles of the output
-  constexpr int kRowBytes = D * 2;
-  extern __shared__ __align__(128) unsigned char dec_smem[];   // K rows [kDecKeys][D] swizzled, then V rows
+  constexpr int kRowBytes = D * 2, kStride = kRowBytes + 16;
+  extern __shared__ __align__(128) unsigned char dec_smem[];   // K rows [kDecKeys], V rows [kDecKeys], Q rows [16]
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int s_fail;
   const int bh = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_keys = a.n_list + a.n_ring;
   const int k_lo = split * kDecKeys, k_hi = min(n_keys, k_lo + kDecKeys), nk = k_hi - k_lo;
   const int b = bh / a.Hkv, hkv = bh % a.Hkv;
-  const uint32_t sK = ptx::smem_u32(dec_smem), sV = sK + kDecKeys * kRowBytes;
+  const uint32_t sK = ptx::smem_u32(dec_smem), sV = sK + kDecKeys * kStride, sQ = sV + kDecKeys * kStride;
+  unsigned char* gQ = dec_smem + 2 * kDecKeys * kStride;
   // The merge kernel is launched as a programmatic dependent of this one: its CTAs may be scheduled from here
   // on and wait (griddepcontrol.wait) until this grid has completed and its stores are visible.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  // Nothing in this call writes the status word but this store (no wait here can expire).
-  if (tid == 0 && split == 0 && bh == 0) *a.status = 0;
-  // chunk c of row r sits at chunk (c & ~7) | ((c ^ r) & 7)
-  auto swz = [](int r, int c) { return (uint32_t)(r * kRowBytes + (((c & ~7) | ((c ^ r) & 7)) << 4)); };
-
+  if (tid == 0) {
+    s_fail = 0;
+    ptx::mbar_init(ptx::smem_u32(&bar), 1);
+    ptx::fence_barrier_init();
+    ptx::mbar_expect_tx(ptx::smem_u32(&bar), (uint32_t)nk * kRowBytes * 2);   // every row copy below reports here
+    // the only writer of the status word before a wait below can expire (seconds later)
+    if (split == 0 && bh == 0) *a.status = 0;
+  }
+  __syncthreads();
   {
     // this thread's row of K and of V
     const int r = tid;
@@ -162,42 +170,58 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const Decod
         const size_t off = ((size_t)bh * 2 * a.L + (a.ring0 + (k - a.n_list)) % (2 * a.L)) * D;
         ks = a.k_ring + off; vs = a.v_ring + off;
       }
-#pragma unroll
-      for (int c = 0; c < CPR; ++c) {
-        cp_async16(sK + swz(r, c), ks + c * 8);
-        cp_async16(sV + swz(r, c), vs + c * 8);
-      }
+      bulk_load(sK + r * kStride, ks, kRowBytes, ptx::smem_u32(&bar));
+      bulk_load(sV + r * kStride, vs, kRowBytes, ptx::smem_u32(&bar));
     } else {
       // rows beyond the split's keys: their probabilities are zero, their V must not be NaN
 #pragma unroll
       for (int c = 0; c < CPR; ++c) {
-        *reinterpret_cast<uint4*>(dec_smem + swz(r, c)) = make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(dec_smem + kDecKeys * kRowBytes + swz(r, c)) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(dec_smem + r * kStride + c * 16) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(dec_smem + (kDecKeys + r) * kStride + c * 16) = make_uint4(0, 0, 0, 0);
       }
     }
-    asm volatile("cp.async.commit_group;" ::: "memory");
   }
 
   const int row = lane >> 2, cpair = (lane & 3) * 2;   // fragment coordinates of this lane
   for (int g0 = 0; g0 < a.G; g0 += kDecHeads) {
     const int ng = min(kDecHeads, a.G - g0);
-    // Q as A fragments: rows = heads g0 + row and g0 + row + 8, straight from global memory
-    uint32_t qa[KS][4];
-    {
-      const __nv_bfloat16* qb = a.q + ((size_t)(b * a.Hq + hkv * a.G + g0)) * D;
-#pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
-        const int c0 = ks * 16 + cpair;
-        qa[ks][0] = row < ng ? *reinterpret_cast<const uint32_t*>(qb + (size_t)row * D + c0) : 0u;
-        qa[ks][1] = row + 8 < ng ? *reinterpret_cast<const uint32_t*>(qb + (size_t)(row + 8) * D + c0) : 0u;
-        qa[ks][2] = row < ng ? *reinterpret_cast<const uint32_t*>(qb + (size_t)row * D + c0 + 8) : 0u;
-        qa[ks][3] = row + 8 < ng ? *reinterpret_cast<const uint32_t*>(qb + (size_t)(row + 8) * D + c0 + 8) : 0u;
-      }
+    // Q of this pass: 16 rows (heads g0 ..., zero beyond the group) into shared memory, 16 bytes per thread and step
+    for (int i = tid; i < kDecHeads * CPR; i += kDecThreads) {
+      const int g = i / CPR, cch = i % CPR;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (g < ng) v = *reinterpret_cast<const uint4*>(a.q + ((size_t)(b * a.Hq + hkv * a.G + g0 + g)) * D + cch * 8);
+      *reinterpret_cast<uint4*>(gQ + g * kStride + cch * 16) = v;
     }
     if (g0 == 0) {
-      asm volatile("cp.async.wait_all;" ::: "memory");
-      __syncthreads();
+      // bounded wait for the copies; a CTA that gives up records it, waits once more for its copies (they write
+      // this CTA's shared memory) and leaves its partial result empty
+      bool got = ptx::mbar_try_wait(ptx::smem_u32(&bar), 0);
+      const long long t0 = clock64();
+      while (!got) {
+        got = ptx::mbar_try_wait(ptx::smem_u32(&bar), 0);
+        if (!got && clock64() - t0 > 4000000000LL) { s_fail = 1; break; }
+      }
     }
+    __syncthreads();
+    if (s_fail) {
+      if (tid == 0) {
+        atomicExch(a.status, (int)LRSA_ERR_TIMEOUT);
+        const long long t0 = clock64();
+        while (!ptx::mbar_try_wait(ptx::smem_u32(&bar), 0) && clock64() - t0 < 4000000000LL) {}
+      }
+      __syncthreads();
+      // empty partial results: maximum -inf, the merge kernel skips them
+      for (int i = tid; i < ng; i += kDecThreads) {
+        float* dst = a.part + (((size_t)bh * a.n_split + split) * a.G + g0 + i) * (D + 2);
+        dst[D] = -INFINITY; dst[D + 1] = 0.f;
+      }
+      continue;
+    }
+    // Q as A fragments: matrices (heads 0-7, channels k..k+7), (heads 8-15, same), then channels k+8..k+15
+    uint32_t qa[KS][4];
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks)
+      ldmatrix_x4(sQ + ((lane & 7) + 8 * ((lane >> 3) & 1)) * kStride + (2 * ks + (lane >> 4)) * 16, qa[ks]);
     // S = Q K^T for this warp's 32 keys: four tiles of 8 keys
     float s[4][4];
 #pragma unroll
@@ -207,7 +231,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const Decod
 #pragma unroll
       for (int q4 = 0; q4 < CPR / 4; ++q4) {
         uint32_t kb[4];
-        ldmatrix_x4(sK + swz(key, 4 * q4 + (lane >> 3)), kb);
+        ldmatrix_x4(sK + key * kStride + (4 * q4 + (lane >> 3)) * 16, kb);
         mma_16816(s[j], qa[2 * q4], kb[0], kb[1]);
         mma_16816(s[j], qa[2 * q4 + 1], kb[2], kb[3]);
       }
@@ -251,14 +275,14 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const Decod
     for (int nt = 0; nt < NT; ++nt) {
       o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
       uint32_t vb[4];
-      ldmatrix_x4_trans(sV + swz(warp * 32 + lane, nt), vb);
+      ldmatrix_x4_trans(sV + (warp * 32 + lane) * kStride + nt * 16, vb);
       mma_16816(o[nt], pa[0], vb[0], vb[1]);
       mma_16816(o[nt], pa[1], vb[2], vb[3]);
     }
     // merge the four warps through shared memory (the K rows are no longer needed once every warp is here;
     // with more than one pass over the heads they are needed again, so the merge buffer then follows V)
     __syncthreads();
-    float* mrg = reinterpret_cast<float*>(dec_smem + (a.G > kDecHeads ? 2 * kDecKeys * kRowBytes : 0));
+    float* mrg = reinterpret_cast<float*>(dec_smem + (a.G > kDecHeads ? (2 * kDecKeys + kDecHeads) * kStride : 0));
     float* mo = mrg;                                   // [4 warps][16 heads][D]
     float* mm_ = mrg + 4 * kDecHeads * D;              // [4][16] maxima
     float* ml = mm_ + 4 * kDecHeads;                   // [4][16] sums
@@ -501,7 +525,7 @@ int lrsa_attn_decode(const lrsa_params_t* params, const void* cache, size_t cach
   const dim3 grid(a.n_split, a.BHkv);
   // K and V rows; the merge buffer (4 warps x 16 heads x (d + 2) floats) lies over them, or behind them when the
   // group has more than 16 query heads and the rows are read again
-  const size_t rows_bytes = (size_t)2 * kDecKeys * g.d * sizeof(__nv_bfloat16);
+  const size_t rows_bytes = (size_t)(2 * kDecKeys + kDecHeads) * (g.d * sizeof(__nv_bfloat16) + 16);   // K, V and Q rows, padded
   const size_t merge_bytes = (size_t)4 * kDecHeads * (g.d + 2) * sizeof(float);
   const size_t smem = g.G > kDecHeads ? rows_bytes + merge_bytes : (rows_bytes > merge_bytes ? rows_bytes : merge_bytes);
   if (g.d == 128) {
