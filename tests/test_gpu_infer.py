@@ -20,6 +20,9 @@ CASES = [
     (W("i_gqa7", 1, 7, 1, 3 + 4 * 200 + 50, 128, 200, 50, 3, seed=83, values="channel_offset"), (250, 1, 1, 199, 403)),
     (W("i_nosink", 1, 2, 2, 6 * 96, 64, 96, 24, 0, seed=84), (96, 96, 1, 95, 200)),
     (W("i_prefill_once", 1, 4, 2, 4 + 7 * 128 + 3, 128, 128, 64, 4, seed=85), (4 + 7 * 128 + 3,)),
+    # more query heads per KV head than one pass of the decode kernel takes (16): two passes over the keys
+    (W("i_gqa20", 1, 20, 1, 4 + 3 * 128 + 50, 128, 128, 32, 4, seed=88), (200, 1, 150, 87)),
+    (W("i_gqa40_d64", 2, 40, 1, 2 + 3 * 64 + 9, 64, 64, 16, 2, seed=89), (100, 1, 1, 101)),
     # lag windows beyond 4096 tokens are scored by the one-slice-per-CTA kernel, here on the ring
     (W("i_long_window", 1, 2, 1, 2 + 3 * 4608 + 100, 64, 4608, 100, 2, seed=86), (5000, 4608, 1, 4000)),
 ]
