@@ -172,3 +172,40 @@ def test_cfg5_sweep_index_agreement_all_points():
 @pytest.mark.parametrize("point", [0, 3, 16, 19])
 def test_cfg5_sweep_attention_corners(point):
     _run_full(workloads.sweep_points()[point], 16, 2, 1)
+
+
+@pytest.mark.parametrize("wname,ndp", [("CFG1", 1), ("CFG2", 1), ("CFG2", 0), ("CFG3", 1)])
+def test_every_element_against_the_cuda_core_kernels(wname, ndp):
+    """The oracle reaches only sampled rows at these sizes.  Every element of O, LSE, dQ, dK and dV is therefore
+    also compared with the library's second implementation of the same calls: CUDA-core kernels, one warp per
+    row, fp32 throughout, no tiles, no tensor memory, no pipelines (and themselves checked against the oracle on
+    small shapes in test_gpu_parity).  A tile that went wrong anywhere - a ragged edge, a diagonal, a hand-off -
+    shows as an error of order one.  Two implementations that each hold the contract differ by at most twice its
+    bound, which is the bound used here; the comparison runs on the GPU (torch elementwise ops on the outputs)."""
+    w = getattr(workloads, wname)
+    host = workloads.generate(w)
+    dev = {k: v.cuda() for k, v in host.items()}
+    p = lrsa.Params.from_workload(w, n_dense_prev=ndp)
+    idx, _ = lrsa.lrsa_score_select(p, dev["K"], dev["V"])
+    outs = []
+    for impl in (0, 1):
+        lrsa.lrsa_debug_set_impl(impl)
+        try:
+            wsb = lrsa.lrsa_workspace_bytes(p)
+            ws1, ws2 = lrsa.new_workspace(wsb[1]), lrsa.new_workspace(wsb[2])
+            O, LSE = lrsa.lrsa_attn_fwd(p, dev["Q"], dev["K"], dev["V"], idx, workspace=ws1)
+            dQ, dK, dV = lrsa.lrsa_attn_bwd(p, dev["Q"], dev["K"], dev["V"], O, dev["dO"], LSE, idx, workspace=ws2)
+            torch.cuda.synchronize()
+            assert lrsa.lrsa_workspace_status(ws1) == 0 and lrsa.lrsa_workspace_status(ws2) == 0
+            outs.append(dict(O=O, LSE=LSE, dQ=dQ, dK=dK, dV=dV))
+        finally:
+            lrsa.lrsa_debug_set_impl(0)
+    for name in ("O", "LSE", "dQ", "dK", "dV"):
+        a, b = outs[0][name].float(), outs[1][name].float()
+        assert torch.isfinite(a).all(), name
+        err = (a - b).abs()
+        bound = 2.0 * (2e-3 if name == "LSE" else 2e-2 + 2.0 ** -8 * b.abs())
+        worst = (err / bound).max().item()
+        print(f"{wname} ndp={ndp} {name}: {err.numel()} elements, max |difference| {err.max().item():.3g}, "
+              f"worst difference/bound {worst:.3g}")
+        assert worst <= 1.0, (name, worst)
