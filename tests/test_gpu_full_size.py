@@ -174,14 +174,20 @@ def test_cfg5_sweep_attention_corners(point):
     _run_full(workloads.sweep_points()[point], 16, 2, 1)
 
 
-@pytest.mark.parametrize("wname,ndp", [("CFG1", 1), ("CFG2", 1), ("CFG2", 0), ("CFG3", 1)])
+@pytest.mark.parametrize("wname,ndp", [("CFG1", 1), ("CFG2", 1), ("CFG2", 0), ("CFG3", 1), ("CFG4", 1)])
 def test_every_element_against_the_cuda_core_kernels(wname, ndp):
     """The oracle reaches only sampled rows at these sizes.  Every element of O, LSE, dQ, dK and dV is therefore
     also compared with the library's second implementation of the same calls: CUDA-core kernels, one warp per
     row, fp32 throughout, no tiles, no tensor memory, no pipelines (and themselves checked against the oracle on
     small shapes in test_gpu_parity).  A tile that went wrong anywhere - a ragged edge, a diagonal, a hand-off -
     shows as an error of order one.  Two implementations that each hold the contract differ by at most twice its
-    bound, which is the bound used here; the comparison runs on the GPU (torch elementwise ops on the outputs)."""
+    bound, which is the bound used here; the comparison runs on the GPU (torch elementwise ops on the outputs).
+    Config 4 (a hundredth of the keys eight times larger, seen by up to 130 000 queries each) is held to that
+    bound for O and LSE only: its gradient elements are cancelling sums of very many large terms, for which
+    neither implementation holds an absolute bound (the CUDA-core kernels take D = rowsum(dO * O) from the bf16 O,
+    the tensor-core kernels round P and dS to bf16: 2^-9 of the sum of the absolute terms either way, see
+    test_attention_fwd_bwd's ill-conditioned case); there the relative L2 difference is asserted and the
+    element-wise figures are printed."""
     w = getattr(workloads, wname)
     host = workloads.generate(w)
     dev = {k: v.cuda() for k, v in host.items()}
@@ -206,6 +212,11 @@ def test_every_element_against_the_cuda_core_kernels(wname, ndp):
         err = (a - b).abs()
         bound = 2.0 * (2e-3 if name == "LSE" else 2e-2 + 2.0 ** -8 * b.abs())
         worst = (err / bound).max().item()
+        rel = (err.double().pow(2).sum() / b.double().pow(2).sum()).sqrt().item()
+        over = (err > bound).sum().item()
         print(f"{wname} ndp={ndp} {name}: {err.numel()} elements, max |difference| {err.max().item():.3g}, "
-              f"worst difference/bound {worst:.3g}")
-        assert worst <= 1.0, (name, worst)
+              f"worst difference/bound {worst:.3g}, {over} above the bound, relative L2 {rel:.3g}")
+        if wname == "CFG4" and name in ("dQ", "dK", "dV"):
+            assert rel <= 1e-2, (name, rel)
+        else:
+            assert worst <= 1.0, (name, worst)
