@@ -196,13 +196,20 @@ __device__ void select_window(const ScoreArgs& a, int bh, int w, unsigned char* 
         while (above + c[j] < (uint32_t)remaining) { above += c[j]; ++j; }
         ibuf[0] = 255 - 8 * lane - j;
         ibuf[1] = remaining - (int)above;
+        ibuf[2] = (int)c[j];   // keys in the chosen bin
       }
     }
     scoring_warps_sync();
     prefix |= (uint32_t)ibuf[0] << shift;
     mask |= 255u << shift;
     remaining = ibuf[1];
+    // Every key of the chosen bin is kept: the remaining bits need not be resolved.  (With 8-bit digits a
+    // thousand keys are alone in their bin after two passes, so this ends the search at half its length.)
+    // The threshold is then the bin's lowest possible key: keys above it are kept as "greater", keys equal to
+    // it as "equal", of which `remaining` is at least as many as exist.
+    const bool whole_bin = ibuf[2] == remaining;
     scoring_warps_sync();
+    if (whole_bin) break;
   }
   const uint32_t kth = prefix;    // K-th largest key
   const int need_eq = remaining;  // how many keys equal to it are kept (lowest positions first)
